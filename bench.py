@@ -742,8 +742,8 @@ def run_timeline(args, wl):
         raise RuntimeError("the timeline needs a CUDA device")
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    build.build()
-    binding.load()
+    build.build_trace()
+    binding.select_trace_build()      # the stamps exist only in the developer build of the library
     r = StepRunner(wl, dev)
     for _ in range(2):
         r.draft_phase(); r.verify_phase(); r.tail_phase()

@@ -22,8 +22,9 @@
  *     negative values are the MASW_E* codes below and masw_last_error() describes the failure.
  *   - Device-side conditions that the host cannot see in advance (a full slot region, a wait on one of
  *     the kernel's own copies that ran out) never trap: the kernel records a bit in a status word,
- *     skips the offending access and returns.  mem_get_state reads the word back; accept_reject takes
- *     its own status pointer.
+ *     skips the offending access and returns.  mem_get_state reads the draft memory's word back;
+ *     verify_attend and accept_reject take a status pointer of their own.  After MASW_STATUS_WAIT_TIMEOUT
+ *     the outputs of that launch are meaningless; the next launch on the same workspace is sound again.
  *   - There is no CPU fallback: without a CUDA device every compute entry point fails with MASW_ECUDA.
  *
  * Positions are 0-based: the paper's token i (1-based) is index i-1.
@@ -51,7 +52,8 @@ enum {
 enum {
   MASW_STATUS_SLOT_OVERFLOW = 1,   /* a slot append was skipped: slot region full */
   MASW_STATUS_WAIT_TIMEOUT = 2,    /* a bounded wait on the kernel's own bulk copies gave up */
-  MASW_STATUS_BAD_LOGIT = 4,       /* accept_reject met a NaN logit or |logit / temperature| too large */
+  MASW_STATUS_BAD_LOGIT = 4,       /* accept_reject met a NaN or infinite logit (a -inf mask included), or, when sampling,
+                                      |logit / temperature| too large */
   MASW_STATUS_BAD_TOKEN = 8        /* accept_reject met a draft token outside [0, V) */
 };
 
@@ -91,7 +93,18 @@ typedef struct masw_kv_desc {
   int32_t capacity;          /* entries allocated per (sequence, head) */
   const int32_t* kv_len;     /* [device] [batch] entries in use, INCLUDING the T rows being verified */
   float softmax_scale;       /* 0 selects 1 / sqrt(D) */
+  int32_t flags;             /* MASW_KV_* bits, 0 for the defaults */
+  int32_t* status;           /* [device] one int32 that receives MASW_STATUS_* bits (OR-ed in), or NULL */
 } masw_kv_desc;
+
+/* masw_kv_desc.flags / masw_paged_kv_desc.flags */
+enum {
+  /* verify_attend, head_dim 128: assign every KV tile to its split statically instead of letting the splits
+   * of a head claim tiles from a shared pool.  A repeated call on the same inputs then returns the same
+   * bits (the pooled schedule only agrees within the rounding of the bf16 probabilities), a little slower
+   * because every split waits for the slowest SM. */
+  MASW_KV_DETERMINISTIC = 1
+};
 
 /* ---------------------------------------------------------------------------------------------------
  * Sizing.  Host only, no CUDA call.
@@ -120,7 +133,8 @@ int mem_load(masw_mem* mem, int layer, int region, const void* k, const void* v,
 
 /* Sets / reads the per-sequence counters: t[b] = committed raw tokens, n_slots[b] = committed slots.
  * Host arrays of length batch.  mem_set_state enqueues on `stream`; mem_get_state synchronises
- * `stream` and also returns the status word (any of t, n_slots, status may be NULL). */
+ * `stream` and also returns the status word (any of t, n_slots, status may be NULL).  Status bits
+ * accumulate on the device between reads; a read with status != NULL returns them and clears the word. */
 int mem_set_state(masw_mem* mem, const int32_t* t /*[host]*/, const int32_t* n_slots /*[host]*/, void* stream);
 int mem_get_state(masw_mem* mem, int32_t* t /*[host]*/, int32_t* n_slots /*[host]*/, int32_t* status /*[host]*/, void* stream);
 
@@ -164,7 +178,7 @@ int mem_rollback(masw_mem* mem, const int32_t* t_keep, const int32_t* slots_keep
  * the last row is the memory-slot token inserted after the last raw row: it sees what that raw row
  * sees plus its own pending slot entry.  Outputs: o [device] fp32 [batch][n_q][Hq][D];
  * lse [device] fp32 [batch][n_q][Hq] (natural-log sum of exp of the scaled scores) or NULL;
- * o_bf16 [device] bf16 copy of o or NULL.  n_q * (Hq/Hkv) must be <= 16. */
+ * o_bf16 [device] bf16 copy of o or NULL.  n_q * (Hq/Hkv) must be <= 64 (and n_q - last_row_is_slot <= gamma_max). */
 int draft_attend(masw_mem* mem, int layer, const void* q, int n_q, int last_row_is_slot,
                  float* o, float* lse, void* o_bf16, void* stream);
 
@@ -234,6 +248,8 @@ typedef struct masw_paged_kv_desc {
   int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128 */
   const int32_t* kv_len;     /* [device] [batch] entries in use, INCLUDING the T rows being verified; <= 128 max_pages */
   float softmax_scale;       /* 0 selects 1 / sqrt(D) */
+  int32_t flags;             /* MASW_KV_* bits, 0 for the defaults */
+  int32_t* status;           /* [device] one int32 that receives MASW_STATUS_* bits (OR-ed in), or NULL */
 } masw_paged_kv_desc;
 
 /* Scratch bytes for verify_attend_paged (same rules as verify_workspace_bytes).  Host only. */
@@ -259,7 +275,9 @@ size_t accept_workspace_bytes(int batch, int gamma, int vocab);
  *   replacement is drawn from norm(max(0, p_n - q_n)); with no rejection the bonus is drawn from
  *   p_gamma; the final draw always uses uniforms[b][gamma].  Probabilities are 40-bit fixed-point
  *   integer weights and all comparisons are exact integer arithmetic, so decisions are reproducible
- *   bit for bit on any conforming implementation.
+ *   bit for bit on any conforming implementation.  The sums of those weights are kept in 64 bits, which
+ *   holds for vocab <= 131071 (the worst case, p and q flat on disjoint halves of the vocabulary, sums to
+ *   vocab^2 2^30): a larger vocabulary is refused with MASW_EINVAL when temperature > 0.
  * Outputs: n_accepted [device] int32 [batch]; out_tokens [device] int32 [batch][gamma+1], unused = -1;
  * status [device] int32 or NULL receives MASW_STATUS_BAD_* bits (OR-ed in). */
 int accept_reject(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libmasw.so")
 MASW_OK, MASW_EINVAL, MASW_EALIGN, MASW_ECAPACITY, MASW_ESTATE, MASW_ECUDA = 0, -1, -2, -3, -4, -5
 STATUS_SLOT_OVERFLOW, STATUS_WAIT_TIMEOUT, STATUS_BAD_LOGIT, STATUS_BAD_TOKEN = 1, 2, 4, 8
 REGION_SINK, REGION_SLOT, REGION_LOCAL = 0, 1, 2
+KV_DETERMINISTIC = 1
 
 EXPORTED_SYMBOLS = [
     "masw_sizes", "mem_init", "mem_free", "mem_load", "mem_set_state", "mem_get_state", "mem_update",
@@ -41,7 +42,8 @@ class masw_config(C.Structure):
 class masw_kv_desc(C.Structure):
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64),
                 ("stride_n", C.c_int64), ("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
-                ("head_dim", C.c_int32), ("capacity", C.c_int32), ("kv_len", C.c_void_p), ("softmax_scale", C.c_float)]
+                ("head_dim", C.c_int32), ("capacity", C.c_int32), ("kv_len", C.c_void_p), ("softmax_scale", C.c_float),
+                ("flags", C.c_int32), ("status", C.c_void_p)]
 
 
 _lib = None
@@ -50,13 +52,17 @@ _lib = None
 def load() -> C.CDLL:
     """Load libmasw.so (built in-tree by paper_2608_30252_b200.build); raises if it is missing."""
     global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(LIB_PATH):
+    if _lib is None:
+        _lib = _open(LIB_PATH)
+    return _lib
+
+
+def _open(path) -> C.CDLL:
+    if not os.path.exists(path):
         raise FileNotFoundError(
-            f"{LIB_PATH} not found: build it with `python -m paper_2608_30252_b200.build` "
+            f"{path} not found: build it with `python -m paper_2608_30252_b200.build` "
             "(there is no CPU fallback)")
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
     lib.masw_sizes.argtypes = [C.POINTER(masw_config), C.POINTER(sz), C.POINTER(sz)]
     lib.mem_init.argtypes = [C.POINTER(masw_config), vp, sz, vp, sz, vp, C.POINTER(vp)]
@@ -86,7 +92,6 @@ def load() -> C.CDLL:
     for name in ("masw_sizes", "mem_init", "mem_load", "mem_set_state", "mem_get_state", "mem_update", "mem_advance",
                  "mem_rollback", "draft_attend", "draft_append_attend", "draft_boundary_attend", "verify_attend", "accept_reject"):
         getattr(lib, name).restype = C.c_int
-    _lib = lib
     return lib
 
 
@@ -144,9 +149,9 @@ def masw_sizes(cfg: MaswConfig):
 class DraftMemory:
     """Owns the device buffers (torch) and the library handle of one draft memory."""
 
-    def __init__(self, cfg: MaswConfig, device="cuda"):
+    def __init__(self, cfg: MaswConfig, device="cuda", lib=None):
         self.cfg = cfg
-        self.lib = load()
+        self.lib = lib or load()
         self.device = torch.device(device)
         arena_bytes, ws_bytes = masw_sizes(cfg)
         self.arena = torch.empty(arena_bytes, dtype=torch.uint8, device=self.device)
@@ -297,12 +302,12 @@ DraftMemory.draft_prefill_slots = _draft_prefill_slots
 DraftMemory.draft_prefill_attend = _draft_prefill_attend
 
 
-def _kv_desc(k, v, kv_len, n_q_heads, softmax_scale=0.0) -> masw_kv_desc:
+def _kv_desc(k, v, kv_len, n_q_heads, softmax_scale=0.0, flags=0, status=None) -> masw_kv_desc:
     assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.stride() == v.stride() and k.stride(-1) == 1
-    assert kv_len.dtype == torch.int32
+    assert kv_len.dtype == torch.int32 and (status is None or status.dtype == torch.int32)
     B, Hkv, cap, D = k.shape
     return masw_kv_desc(k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2), B, n_q_heads, Hkv, D, cap,
-                        kv_len.data_ptr(), softmax_scale)
+                        kv_len.data_ptr(), softmax_scale, flags, None if status is None else status.data_ptr())
 
 
 def verify_workspace(k, kv_len, n_q_heads, T) -> torch.Tensor:
@@ -312,30 +317,33 @@ def verify_workspace(k, kv_len, n_q_heads, T) -> torch.Tensor:
     return torch.zeros(n, dtype=torch.uint8, device=k.device)
 
 
-def verify_attend(k, v, kv_len, q, workspace=None, out=None, lse=None, out_bf16=None, softmax_scale=0.0):
-    """k, v: bf16 [B, Hkv, cap, D] views; kv_len int32 [B] (including the T rows); q bf16 [B, T, Hq, D]."""
+def verify_attend(k, v, kv_len, q, workspace=None, out=None, lse=None, out_bf16=None, softmax_scale=0.0,
+                  deterministic=False, status=None, lib=None):
+    """k, v: bf16 [B, Hkv, cap, D] views; kv_len int32 [B] (including the T rows); q bf16 [B, T, Hq, D].
+    deterministic: static tile schedule (bitwise repeatable); status: int32 [1] device tensor for MASW_STATUS_* bits."""
     assert q.dtype == torch.bfloat16 and q.is_contiguous()
     B, T, Hq, D = q.shape
-    desc = _kv_desc(k, v, kv_len, Hq, softmax_scale)
+    desc = _kv_desc(k, v, kv_len, Hq, softmax_scale, KV_DETERMINISTIC if deterministic else 0, status)
     if workspace is None:
         workspace = verify_workspace(k, kv_len, Hq, T)
     if out is None:
         out = torch.empty((B, T, Hq, D), dtype=torch.float32, device=q.device)
     if lse is None:
         lse = torch.empty((B, T, Hq), dtype=torch.float32, device=q.device)
-    _check(load().verify_attend(C.byref(desc), _ptr(q), T, _ptr(out), _ptr(lse), _ptr(out_bf16), _ptr(workspace),
-                                workspace.numel(), _stream()))
+    _check((lib or load()).verify_attend(C.byref(desc), _ptr(q), T, _ptr(out), _ptr(lse), _ptr(out_bf16), _ptr(workspace),
+                                         workspace.numel(), _stream()))
     return out, lse
 
 
 class masw_paged_kv_desc(C.Structure):
     _fields_ = [("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("page_table", C.c_void_p), ("n_pages", C.c_int32),
                 ("max_pages", C.c_int32), ("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
-                ("head_dim", C.c_int32), ("kv_len", C.c_void_p), ("softmax_scale", C.c_float)]
+                ("head_dim", C.c_int32), ("kv_len", C.c_void_p), ("softmax_scale", C.c_float), ("flags", C.c_int32),
+                ("status", C.c_void_p)]
 
 
 def verify_attend_paged(k_pages, v_pages, page_table, kv_len, q, workspace=None, out=None, lse=None, out_bf16=None,
-                        softmax_scale=0.0):
+                        softmax_scale=0.0, deterministic=False, status=None):
     """k_pages, v_pages: bf16 [n_pages, Hkv, 128, D] contiguous; page_table int32 [B, max_pages]; kv_len int32 [B]
     (including the T rows); q bf16 [B, T, Hq, D].  Returns (o fp32, lse fp32, workspace)."""
     assert k_pages.dtype == torch.bfloat16 and k_pages.is_contiguous() and v_pages.is_contiguous() and k_pages.shape == v_pages.shape
@@ -345,7 +353,8 @@ def verify_attend_paged(k_pages, v_pages, page_table, kv_len, q, workspace=None,
     assert page == 128
     B, T, Hq, _ = q.shape
     desc = masw_paged_kv_desc(k_pages.data_ptr(), v_pages.data_ptr(), page_table.data_ptr(), n_pages, page_table.shape[1], B, Hq,
-                              Hkv, D, kv_len.data_ptr(), softmax_scale)
+                              Hkv, D, kv_len.data_ptr(), softmax_scale, KV_DETERMINISTIC if deterministic else 0,
+                              None if status is None else status.data_ptr())
     lib = load()
     lib.verify_paged_workspace_bytes.argtypes = [C.POINTER(masw_paged_kv_desc), C.c_int]
     lib.verify_paged_workspace_bytes.restype = C.c_size_t
@@ -412,12 +421,40 @@ def accept_reject_static(target_logits, draft_logits, draft_tokens, uniforms, te
     return n_accepted, out_tokens
 
 
-def debug_set_trace(buffer) -> None:
-    """Developer hook (not part of the C ABI header): while `buffer` (an int64 CUDA tensor of at least
-    16 words per CTA of the next launches) is set, the attention kernels write a few %globaltimer
-    stamps per CTA into it.  Pass None to switch the stamps off again."""
-    lib = load()
-    lib.masw_debug_set_trace.argtypes = [C.c_void_p]
-    lib.masw_debug_set_trace.restype = None
-    lib.masw_debug_set_trace(C.c_void_p(buffer.data_ptr()) if buffer is not None else None)
+# ---- developer build (libmasw_trace.so, compiled with -DMASW_TRACE; never loaded by the product path) ----
+TRACE_LIB_PATH = os.path.join(_HERE, "libmasw_trace.so")
+_trace_lib = None
 
+
+def load_trace() -> C.CDLL:
+    """The developer build of the same sources: phase stamps in the attention kernels, a settable limit for
+    their bounded waits and a switch that leaves one tile copy out.  Used by `bench.py --timeline` and by the
+    test of the give-up path; it is a separate library, so the product library carries none of this."""
+    global _trace_lib
+    if _trace_lib is None:
+        lib = _open(TRACE_LIB_PATH)
+        lib.masw_debug_set_trace.argtypes = [C.c_void_p]
+        lib.masw_debug_set_trace.restype = None
+        lib.masw_debug_set_wait.argtypes = [C.c_int, C.c_int]
+        lib.masw_debug_set_wait.restype = None
+        _trace_lib = lib
+    return _trace_lib
+
+
+def select_trace_build() -> None:
+    """Route every call of this module to the developer build (for `bench.py --timeline`; call it first)."""
+    global _lib
+    _lib = load_trace()
+
+
+def debug_set_trace(buffer) -> None:
+    """Developer build: while `buffer` (an int64 CUDA tensor of at least 16 words per CTA of the next launches)
+    is set, the attention kernels of libmasw_trace.so write a few %globaltimer stamps per CTA into it.  Pass
+    None to switch the stamps off again."""
+    load_trace().masw_debug_set_trace(C.c_void_p(buffer.data_ptr()) if buffer is not None else None)
+
+
+def debug_set_wait(wait_limit=0, drop_tile=-1) -> None:
+    """Developer build: polls after which the kernels' bounded waits give up (0 = the normal limit) and the
+    CTA-local index of one tile whose copy is armed but never issued (-1 = none)."""
+    load_trace().masw_debug_set_wait(int(wait_limit), int(drop_tile))

@@ -8,6 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libmasw.so")
+TRACE_LIB_PATH = os.path.join(HERE, "libmasw_trace.so")
 SOURCES = ["api.cu", "attend.cu", "prefill.cu", "mem.cu", "accept.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -22,12 +23,25 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: the MASW library cannot be built")
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB_PATH):
+def needs_build(lib_path: str = None) -> bool:
+    lib_path = lib_path or LIB_PATH
+    if not os.path.exists(lib_path):
         return True
-    lib_mtime = os.path.getmtime(LIB_PATH)
+    lib_mtime = os.path.getmtime(lib_path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "masw.h")]
     return any(os.path.getmtime(d) > lib_mtime for d in deps)
+
+
+def build_trace(force: bool = False) -> str:
+    """Compile the developer build (-DMASW_TRACE: phase stamps, settable wait limit, droppable tile copy) into
+    paper_2608_30252_b200/libmasw_trace.so.  Only `bench.py --timeline` and the give-up test load it."""
+    if not force and not needs_build(TRACE_LIB_PATH):
+        return TRACE_LIB_PATH
+    cmd = [_nvcc(), *NVCC_FLAGS, "-DMASW_TRACE", "-o", TRACE_LIB_PATH] + [os.path.join(CSRC, s) for s in SOURCES]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    return TRACE_LIB_PATH
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

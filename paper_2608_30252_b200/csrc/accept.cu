@@ -281,6 +281,12 @@ accept_reject_kernel(const unsigned short* tl, const unsigned short* dl, const i
 
 }  // namespace masw
 
+namespace masw {
+// Sampling keeps the sum of the residual weights in 64 bits.  Its largest value, reached when p and q are flat
+// on disjoint halves of the vocabulary, is (V / 2)^2 2^32 = V^2 2^30, which fits while V < 2^17.
+constexpr int kMaxSamplingVocab = 131071;
+}  // namespace masw
+
 using namespace masw;
 
 extern "C" size_t accept_workspace_bytes(int batch, int gamma, int vocab) {
@@ -300,6 +306,8 @@ extern "C" int accept_reject(const void* target_logits, const void* draft_logits
   if (temperature > 0.f) {
     MASW_REQUIRE(draft_logits != nullptr && uniforms != nullptr, MASW_EINVAL,
                  "accept_reject: sampling needs draft_logits and uniforms");
+    MASW_REQUIRE(vocab <= kMaxSamplingVocab, MASW_EINVAL,
+                 "accept_reject: sampling keeps 64-bit weight sums, exact only for vocab <= %d (got %d)", kMaxSamplingVocab, vocab);
   }
   MASW_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 15) == 0, MASW_EALIGN, "accept_reject: workspace must be 16-byte aligned");
   const AcceptWs w = accept_ws(batch, gamma);
@@ -329,7 +337,6 @@ constexpr size_t kStaticScratchBytes = kStaticTicketBytes + sizeof(RowInfo) * kS
 // looked up per device with cudaGetSymbolAddress below and that pointer is what the kernel receives.
 static __device__ __align__(256) unsigned char g_accept_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
 static std::mutex g_static_mu;
 static unsigned char* g_static_ptr[kMaxDevices] = {};
 
@@ -365,6 +372,8 @@ extern "C" int accept_reject_static(const void* target_logits, const void* draft
   if (temperature > 0.f) {
     MASW_REQUIRE(draft_logits != nullptr && uniforms != nullptr, MASW_EINVAL,
                  "accept_reject_static: sampling needs draft_logits and uniforms");
+    MASW_REQUIRE(vocab <= kMaxSamplingVocab, MASW_EINVAL,
+                 "accept_reject_static: sampling keeps 64-bit weight sums, exact only for vocab <= %d (got %d)", kMaxSamplingVocab, vocab);
   }
   unsigned char* scratch = nullptr;
   int rc = static_scratch(&scratch);

@@ -9,11 +9,17 @@
 
 namespace masw {
 
-// developer hook (not part of the ABI): when set, every attention CTA records phase timestamps here
+#ifdef MASW_TRACE
+// developer build only (never part of the product library): a device buffer that receives per-CTA phase
+// timestamps, a shortened limit for the kernels' bounded waits, and the index of one tile whose copy is left
+// out so that such a wait runs out (the way the give-up path is tested without any fault)
 static long long* g_trace = nullptr;
-// developer hook: 1 forces verify_attend onto the mma.sync kernel (for A/B comparisons)
-static int g_verify_legacy = 0;
-static int g_debug_flags = 0;   // developer switches: 4 / 8 = no early launch of the draft / verify kernel
+static int g_wait_limit = kWaitLimit;
+static int g_drop_tile = -1;
+static void apply_debug(AttendParams& p) { p.trace = g_trace; p.wait_limit = g_wait_limit; p.drop_tile = g_drop_tile; }
+#else
+static void apply_debug(AttendParams&) {}
+#endif
 
 // One kernel instance: up to splits_max independent CTAs per (sequence, KV head), CT CTAs per SM.
 template <int D, int MT, int EW, int TE, int NSTAGE, int CT>
@@ -21,17 +27,15 @@ static int launch_attend(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendP
                          int tiles_upper, int splits_max, cudaStream_t st) {
   using C = AttendCfg<D, MT, EW, TE, NSTAGE>;
   auto kern = attend_kernel<D, MT, EW, TE, NSTAGE, CT>;
-  static bool configured = false;
-  if (!configured) {
-    MASW_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-    configured = true;
-  }
+  static PerDeviceOnce once;
+  { const int rc = set_smem_once(kern, C::kSmemBytes, once); if (rc != MASW_OK) return rc; }
   int splits = (sm_count() * CT) / (B * Hkv);
   if (splits > splits_max) splits = splits_max;
   if (splits > tiles_upper) splits = tiles_upper;
   if (splits < 1) splits = 1;
   p.splits = splits;
-  p.trace = g_trace;
+  p.wait_limit = kWaitLimit;
+  apply_debug(p);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(splits, Hkv, B);
   cfg.blockDim = dim3(C::kThreads, 1, 1);
@@ -44,7 +48,7 @@ static int launch_attend(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendP
   if (splits > 1) { attr[na].id = cudaLaunchAttributeCooperative; attr[na].val.cooperative = 1; ++na; }
   // the kernel may be set up while its predecessor in the stream drains: it touches no global memory before
   // its griddepcontrol.wait
-  if (!(g_debug_flags & 4)) { attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na; }
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na;
   cfg.attrs = attr;
   cfg.numAttrs = na;
   MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmK, tmV, p));
@@ -58,17 +62,15 @@ static int launch_attend_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, Atte
                             int tiles_upper, int splits_max, cudaStream_t st) {
   using C = TcCfg<NQ, NK, NV>;
   auto kern = attend_tc_kernel<NQ, NK, NV>;
-  static bool configured = false;
-  if (!configured) {
-    MASW_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-    configured = true;
-  }
+  static PerDeviceOnce once;
+  { const int rc = set_smem_once(kern, C::kSmemBytes, once); if (rc != MASW_OK) return rc; }
   int splits = sm_count() / (B * Hkv);
   if (splits > splits_max) splits = splits_max;
   if (splits > tiles_upper) splits = tiles_upper;
   if (splits < 1) splits = 1;
   p.splits = splits;
-  p.trace = g_trace;
+  p.wait_limit = kWaitLimit;
+  apply_debug(p);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(splits, Hkv, B);
   cfg.blockDim = dim3(C::kThreads, 1, 1);
@@ -77,7 +79,7 @@ static int launch_attend_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, Atte
   cudaLaunchAttribute attr[2];
   int na = 0;
   if (splits > 1) { attr[na].id = cudaLaunchAttributeCooperative; attr[na].val.cooperative = 1; ++na; }
-  if (!(g_debug_flags & 8)) { attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na; }
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na;
   cfg.attrs = attr;
   cfg.numAttrs = na;
   MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmK, tmV, p));
@@ -170,9 +172,13 @@ int get_kv_maps(const masw_kv_desc& kv, int box, CUtensorMap* tk, CUtensorMap* t
 
 using namespace masw;
 
+#ifdef MASW_TRACE
 extern "C" void masw_debug_set_trace(void* device_buffer) { g_trace = static_cast<long long*>(device_buffer); }
-extern "C" void masw_debug_set_verify_legacy(int on) { g_verify_legacy = on; }
-extern "C" void masw_debug_set_flags(int flags) { g_debug_flags = flags; }
+extern "C" void masw_debug_set_wait(int wait_limit, int drop_tile) {
+  g_wait_limit = wait_limit > 0 ? wait_limit : kWaitLimit;
+  g_drop_tile = drop_tile;
+}
+#endif
 
 struct SlotInputs {
   const void* h_g = nullptr;
@@ -278,7 +284,7 @@ extern "C" int verify_attend(const masw_kv_desc* kv, const void* q, int T, float
   const VerifyWs w = verify_ws(kv->batch, kv->n_kv_heads, G, kv->head_dim, T);
   MASW_REQUIRE(workspace_bytes >= w.total, MASW_ECAPACITY, "verify_attend: workspace %zu < %zu bytes", workspace_bytes, w.total);
   const int mt = (T * G + 15) / 16;
-  const bool use_tc = (kv->head_dim == 128) && !g_verify_legacy;
+  const bool use_tc = (kv->head_dim == 128);
   CUtensorMap tk, tv;
   int rc = get_kv_maps(*kv, use_tc ? 128 : tile_entries(kv->head_dim, mt), &tk, &tv);
   if (rc != MASW_OK) return rc;
@@ -289,7 +295,8 @@ extern "C" int verify_attend(const masw_kv_desc* kv, const void* q, int T, float
   p.part_o = reinterpret_cast<unsigned long long*>(ws + w.off_part_o);
   p.part_ml = reinterpret_cast<unsigned long long*>(ws + w.off_part_ml);
   p.tickets = reinterpret_cast<int*>(ws + w.off_tickets);
-  p.status = nullptr;
+  p.status = kv->status;
+  p.deterministic = (kv->flags & MASW_KV_DETERMINISTIC) ? 1 : 0;
   p.t = nullptr; p.n_slots = nullptr; p.kv_len = kv->kv_len;
   p.n_q = T; p.last_row_is_slot = 0;
   p.G = G; p.Hq = kv->n_q_heads; p.Hkv = kv->n_kv_heads;
@@ -348,7 +355,8 @@ extern "C" int verify_attend_paged(const masw_paged_kv_desc* kv, const void* q, 
   p.part_o = reinterpret_cast<unsigned long long*>(ws + w.off_part_o);
   p.part_ml = reinterpret_cast<unsigned long long*>(ws + w.off_part_ml);
   p.tickets = reinterpret_cast<int*>(ws + w.off_tickets);
-  p.status = nullptr;
+  p.status = kv->status;
+  p.deterministic = (kv->flags & MASW_KV_DETERMINISTIC) ? 1 : 0;
   p.t = nullptr; p.n_slots = nullptr; p.kv_len = kv->kv_len;
   p.n_q = T; p.last_row_is_slot = 0;
   p.G = G; p.Hq = kv->n_q_heads; p.Hkv = kv->n_kv_heads;

@@ -20,7 +20,6 @@ namespace masw {
 
 constexpr int kMaxSeg = 4;
 constexpr int kMaxSplitsDev = 64;   // upper bound on splits per (sequence, KV head); the host clamps to it
-constexpr int kSpinLimit = 1 << 20; // polls of the arrival counter before a CTA gives up (about a second)
 
 struct AttendParams {
   const __nv_bfloat16* q;  // [B][n_q][Hq][D]
@@ -60,7 +59,13 @@ struct AttendParams {
   int max_pages;
   int splits;
   float scale_log2e;
-  long long* trace;        // developer hook: per-CTA phase timestamps (null in normal operation)
+  int wait_limit;          // polls after which a bounded wait gives up (kWaitLimit in normal operation)
+  int deterministic;       // verify (tcgen05 kernel): every tile assigned statically, results repeat bit for bit
+#ifdef MASW_TRACE
+  long long* trace;        // developer build: per-CTA phase timestamps (null = off)
+  int drop_tile;           // developer build: the copy of this CTA-local tile is armed but never issued (-1 = off),
+                           // which makes a bounded wait run out without any fault
+#endif
 };
 
 struct Segment {
@@ -229,7 +234,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
               all_ok &= r0.ok && r1.ok;
             }
           }
-          for (int it = 0; !all_ok && it < kSpinLimit; ++it) {   // a split that has not published yet
+          for (int it = 0; !all_ok && it < p.wait_limit; ++it) {   // a split that has not published yet
             __nanosleep(20);
             all_ok = true;
 #pragma unroll
@@ -331,7 +336,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
             all_ok &= okv[u];
           }
         }
-        for (int it = 0; !all_ok && it < kSpinLimit; ++it) {   // a split that has not published yet
+        for (int it = 0; !all_ok && it < p.wait_limit; ++it) {   // a split that has not published yet
           __nanosleep(20);
           all_ok = true;
 #pragma unroll
@@ -460,15 +465,10 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const int b = blockIdx.z;
   const int n_rows = p.n_q * p.G;  // real query rows of this KV head
 
+#ifdef MASW_TRACE
   long long* tr = p.trace ? p.trace + (static_cast<size_t>((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)) * 16 : nullptr;
-  auto stamp = [&](int slot) {
-    if (tr && tid == 0) {
-      long long t;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) : : "memory");
-      tr[slot] = t;
-    }
-  };
-  stamp(0);
+#endif
+  MASW_STAMP(tr, 0);
   const bool is_producer = (tid == C::kConsumerWarps * 32);   // lane 0 of the producer warp
   if (is_producer) {
     prefetch_tensormap(&tmK);   // the descriptor fetches overlap the barrier setup and the counter loads
@@ -543,6 +543,9 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         uint8_t* kdst = pipe + i * C::kStageBytes;
         uint8_t* vdst = kdst + C::kTileBytes;
         mbar_arrive_expect_tx(&full_bar[i], C::kStageBytes);
+#ifdef MASW_TRACE
+        if (i == p.drop_tile) continue;
+#endif
 #pragma unroll
         for (int sub = 0; sub < C::kSub; ++sub)
           tma_load_4d(kdst + sub * C::kSubBytes, &tmK, &full_bar[i], sub * 64, row0, kvh, b, policy);
@@ -594,7 +597,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
   }
   __syncthreads();
-  stamp(1);
+  MASW_STAMP(tr, 1);
 
   const int nseg = plan[0];
   const int tile_begin = plan[1];
@@ -622,11 +625,15 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int row0 = plan[8 + 4 * seg] + i0;
         const int stage = i % NSTAGE;
         const int round = i / NSTAGE;
-        ok = mbar_wait_bounded(&empty_bar[stage], (round - 1) & 1);
+        ok = mbar_wait_bounded(&empty_bar[stage], (round - 1) & 1, p.wait_limit);
         if (!ok) break;
         uint8_t* kdst = pipe + stage * C::kStageBytes;
         uint8_t* vdst = kdst + C::kTileBytes;
         mbar_arrive_expect_tx(&full_bar[stage], C::kStageBytes);
+        plan[5] = i + 1;  // tiles issued so far (read only on the give-up path)
+#ifdef MASW_TRACE
+        if (i == p.drop_tile) continue;
+#endif
 #pragma unroll
         for (int sub = 0; sub < C::kSub; ++sub) {
           tma_load_4d(kdst + sub * C::kSubBytes, &tmK, &full_bar[stage], sub * 64, row0, kvh, b, policy);
@@ -635,7 +642,6 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         for (int sub = 0; sub < C::kSub; ++sub) {
           tma_load_4d(vdst + sub * C::kSubBytes, &tmV, &full_bar[stage], sub * 64, row0, kvh, b, policy);
         }
-        plan[5] = i + 1;  // tiles issued so far (read only on the give-up path)
       }
       if (!ok) {
         plan[3] = 1;
@@ -726,7 +732,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
       }
 
-      ok = mbar_wait_bounded(&full_bar[stage], parity);
+      ok = mbar_wait_bounded(&full_bar[stage], parity, p.wait_limit);
       if (!ok) break;
 
       uint8_t* ksm = pipe + stage * C::kStageBytes;
@@ -756,6 +762,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           int which, r, cg;
           put(idx, __ldg(raw_src(idx, which, r, cg)));
         }
+        fence_proxy_async();   // by every lane that wrote: the stage is handed back to the bulk copies later
         __syncwarp();
       }
 
@@ -768,6 +775,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           const int cg = idx % (D / 8);
           *reinterpret_cast<uint4*>(vsm + (cg >> 3) * C::kSubBytes + r * 128 + ((cg & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
+        fence_proxy_async();   // every lane orders its own stores ahead of the next bulk copy into this stage
         __syncwarp();
       }
 
@@ -906,10 +914,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
       // release the stage to the producer
       __syncwarp();
-      if (lane == 0) {
-        if (valid < TE || patched) fence_proxy_async();
-        mbar_arrive(&empty_bar[stage]);
-      }
+      if (lane == 0) mbar_arrive(&empty_bar[stage]);
     }
     if (!ok && lane == 0) {
       plan[3] = 1;
@@ -923,14 +928,14 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   }
 
   __syncthreads();  // every tile consumed (or abandoned): the stages can be reused as merge scratch
-  stamp(2);
+  MASW_STAMP(tr, 2);
   if (plan[3] != 0) {
     // give-up path: a wait ran out.  Let this CTA's copies that are still in flight land (bounded)
     // before shared memory is reused or released; the outputs of this launch are not meaningful.
     if (tid == 0) {
       const int issued = plan[5];
       for (int i = max(0, issued - NSTAGE); i < issued; ++i) {
-        mbar_wait_bounded(&full_bar[i % NSTAGE], (i / NSTAGE) & 1);
+        mbar_wait_bounded(&full_bar[i % NSTAGE], (i / NSTAGE) & 1, p.wait_limit);
       }
     }
     __syncthreads();
@@ -1053,11 +1058,13 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   }
 
   // ---- cross-split reduction (see split_reduce_and_store)
-  stamp(3);
+  MASW_STAMP(tr, 3);
+#ifdef MASW_TRACE
   if (tr && tid == 0) { tr[5] = 1; tr[6] = n_tiles; unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); tr[7] = sm; }
+#endif
   split_reduce_and_store<D, kRows, C::kThreads>(p, b, kvh, split, n_rows, plan[6], reinterpret_cast<float*>(pipe), tid,
                                                 p.h_g != nullptr ? rope_cs : nullptr);
-  stamp(4);
+  MASW_STAMP(tr, 4);
 }
 
 }  // namespace masw

@@ -187,25 +187,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int n_rows = p.n_q * p.G;
 
+#ifdef MASW_TRACE
   long long* tr = p.trace ? p.trace + (static_cast<size_t>((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)) * 16 : nullptr;
-  auto stamp = [&](int slot) {
-    if (tr && tid == 0) {
-      long long t;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) : : "memory");
-      tr[slot] = t;
-    }
-  };
-  auto stamp_by = [&](int who, int slot) {   // the same from another thread
-    if (tr && tid == who) {
-      long long t;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) : : "memory");
-      tr[slot] = t;
-    }
-  };
-  stamp(0);
+#endif
+  MASW_STAMP(tr, 0);
   // producer state (thread 0 only): the schedule and the pool claim in flight
   constexpr int kStaticNum = 1, kStaticDen = 4;   // share of the tiles that is assigned statically
-  int n_static = 0, n_pool = 0, n_early = 0, pending = 0x7fffffff;
+  int n_static = 0, static_first = 0, n_pool = 0, n_early = 0, pending = 0x7fffffff;
   int* pool_ctr = nullptr;
   // ---- prologue
   if (warp == 1) {
@@ -262,14 +250,25 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // KV head) claim one tile at a time (an atomic counter), so an SM that streams more slowly simply ends up
     // with fewer tiles.  The two counter words alternate with the epoch's parity: this launch uses one, and
     // split 0 clears the other for the next launch, which nobody is using then.
+    // In the deterministic mode there is no pool: every tile is assigned statically (the remainder goes to the
+    // first splits), so each split meets the same tiles in the same order in every launch and the result
+    // repeats bit for bit, at the price of waiting for the slowest SM.
     const int rest = max(0, nt - p.splits);
-    n_static = (rest * kStaticNum / kStaticDen) / p.splits;
-    n_pool = rest - n_static * p.splits;
+    if (p.deterministic) {
+      const int base = rest / p.splits, rem = rest % p.splits;
+      n_static = base + (split < rem ? 1 : 0);
+      n_pool = 0;
+      static_first = p.splits + split * base + min(split, rem);
+    } else {
+      n_static = (rest * kStaticNum / kStaticDen) / p.splits;
+      n_pool = rest - n_static * p.splits;
+      static_first = p.splits + n_pool + split * n_static;
+    }
     const int epoch = __ldcg(p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1));
     pool_ctr = p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + (epoch & 1);
     pending = (n_pool > 0) ? atomicAdd(pool_ctr, 1) : 0x7fffffff;   // used only after the static tiles
     ctl->plan[0] = len;
-    ctl->plan[1] = p.splits + n_pool + split * n_static;
+    ctl->plan[1] = static_first;
     ctl->plan[2] = 0;
     ctl->plan[6] = epoch;
     ctl->error = 0;
@@ -300,7 +299,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   __syncthreads();
   tc_fence_after();
 
-  stamp(1);
+  MASW_STAMP(tr, 1);
   const uint32_t tmem_base = ctl->tmem_base;
   const int kv_total = ctl->plan[0];
   int n_tiles = 0;   // tiles this CTA streamed; each role learns it when it meets the end of the stream
@@ -321,7 +320,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (i < n_res) return ctl->tile_id[i & 15];
         int id = -1;
         if (i - 1 < n_static) {               // index 0 was the first tile, requested in the prologue
-          id = p.splits + n_pool + split * n_static + (i - 1);
+          id = static_first + (i - 1);
         } else if (pending < n_pool) {
           id = p.splits + pending;
           pending = atomicAdd(pool_ctr, 1);   // the next claim is in flight while this tile streams
@@ -335,7 +334,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       int ik = n_early, iv = n_early;   // the first tiles were issued in the prologue
       bool k_done = false, v_done = false;
       int idle = 0;
-      while ((!k_done || !v_done) && idle < kWaitLimit) {
+      while ((!k_done || !v_done) && idle < p.wait_limit) {
         bool progressed = false;
         if (!k_done && (ik < NK || mbar_try_wait(&ctl->k_empty[ik % NK], (ik / NK - 1) & 1))) {
           const int id = resolve(ik);
@@ -347,8 +346,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const bool paged = p.page_table != nullptr;
             const int row0 = paged ? 0 : id * C::kTile, outer = paged ? ctl->page_id[ik & 15] : b;
             mbar_arrive_expect_tx(&ctl->k_full[ik % NK], C::kTileBytes);
-            tma_load_4d(kdst, &tmK, &ctl->k_full[ik % NK], 0, row0, kvh, outer, policy);
-            tma_load_4d(kdst + C::kSubBytes, &tmK, &ctl->k_full[ik % NK], 64, row0, kvh, outer, policy);
+#ifdef MASW_TRACE
+            if (ik != p.drop_tile)
+#endif
+            {
+              tma_load_4d(kdst, &tmK, &ctl->k_full[ik % NK], 0, row0, kvh, outer, policy);
+              tma_load_4d(kdst + C::kSubBytes, &tmK, &ctl->k_full[ik % NK], 64, row0, kvh, outer, policy);
+            }
             ++ik;
           }
           progressed = true;
@@ -388,8 +392,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       for (int i = 0; ok; ++i) {
         {
           const int sb = i & 1;
-          ok = mbar_wait_bounded(&ctl->k_full[i % NK], (i / NK) & 1);
-          if (ok && i >= 2) ok = mbar_wait_bounded(&ctl->s_empty[sb], ((i >> 1) - 1) & 1);
+          ok = mbar_wait_bounded(&ctl->k_full[i % NK], (i / NK) & 1, p.wait_limit);
+          if (ok && i >= 2) ok = mbar_wait_bounded(&ctl->s_empty[sb], ((i >> 1) - 1) & 1, p.wait_limit);
           if (!ok) break;
           if (ctl->tile_id[i & 15] < 0) {
             n_end = i;
@@ -409,8 +413,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         if (i >= 1) {
           const int j = i - 1;
-          ok = mbar_wait_bounded(&ctl->p_full[j & 1], (j >> 1) & 1);
-          if (ok) ok = mbar_wait_bounded(&ctl->v_full[j % NV], (j / NV) & 1);
+          ok = mbar_wait_bounded(&ctl->p_full[j & 1], (j >> 1) & 1, p.wait_limit);
+          if (ok) ok = mbar_wait_bounded(&ctl->v_full[j % NV], (j / NV) & 1, p.wait_limit);
           if (!ok) break;
           tc_fence_after();
           const uint32_t v_base = smem_u32(v_ring + (j % NV) * C::kTileBytes);
@@ -454,7 +458,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     volatile int* stop = &ctl->stop[grp];
     for (int i = 0;; ++i) {
       const int sb = i & 1;
-      if (ok) ok = mbar_wait_bounded(&ctl->s_full[sb], (i >> 1) & 1);
+      if (ok) ok = mbar_wait_bounded(&ctl->s_full[sb], (i >> 1) & 1, p.wait_limit);
       ok = __all_sync(0xffffffffu, ok);
       const int tile = ctl->tile_id[i & 15];
       // The loop ends for the whole group at the named barrier below: at the end-of-stream marker, or
@@ -538,9 +542,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
       // the P tile is double-buffered: tile i - 2's P.V must be complete before its buffer is reused;
       // only a moved maximum has to wait for tile i - 1's P.V, to rescale O^T in tensor memory
-      if (i >= 2 && ok) ok = mbar_wait_bounded(&ctl->p_empty[i & 1], ((i >> 1) - 1) & 1);
+      if (i >= 2 && ok) ok = mbar_wait_bounded(&ctl->p_empty[i & 1], ((i >> 1) - 1) & 1, p.wait_limit);
       if (i > 0 && any_changed) {
-        if (ok) ok = mbar_wait_bounded(&ctl->o_ready, (i - 1) & 1);
+        if (ok) ok = mbar_wait_bounded(&ctl->o_ready, (i - 1) & 1, p.wait_limit);
         ok = __all_sync(0xffffffffu, ok);   // the tensor-memory accesses below are warp-wide
         tc_fence_after();
         if (ok) {
@@ -570,7 +574,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       // entries beyond the cache length hold foreign bytes: zero their V rows (their probability is 0,
       // but 0 x non-finite would poison the accumulator); the first group does it
       if (grp == 0 && (tile + 1) * C::kTile > kv_total) {   // only the last tile of the cache can have such rows
-        if (ok) ok = mbar_wait_bounded(&ctl->v_full[i % NV], (i / NV) & 1);   // the tile must have landed before it is patched
+        if (ok) ok = mbar_wait_bounded(&ctl->v_full[i % NV], (i / NV) & 1, p.wait_limit);   // the tile must have landed before it is patched
         // rows [valid, 128) are one contiguous range in each 64-column half of the tile (the swizzle
         // permutes inside a row group, and whole rows are cleared); consecutive threads clear
         // consecutive 16-byte chunks, which is free of bank conflicts
@@ -586,7 +590,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       mbar_arrive(&ctl->p_full[i & 1]);
     }
     if (!ok) ctl->error = 1;
-    stamp_by(128, 8);
+    MASW_STAMP_BY(tr, 128, 8);
 
     // ---- epilogue of the softmax warps: this split's partial (o unnormalised, m, l) -> global scratch
     const int bh = b * p.Hkv + kvh;
@@ -595,7 +599,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int tag = ctl->plan[6] + 1;   // this launch's epoch tag
     bool have_o = ok && n_tiles > 0;
     if (have_o) {
-      have_o = mbar_wait_bounded(&ctl->o_ready, (n_tiles - 1) & 1);
+      have_o = mbar_wait_bounded(&ctl->o_ready, (n_tiles - 1) & 1, p.wait_limit);
       tc_fence_after();
     }
     have_o = __all_sync(0xffffffffu, have_o);
@@ -627,12 +631,14 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       rec_store2(pml + r * 2, ctl->mfinal[r], ctl->lsum[0][r] + ctl->lsum[1][r] + ctl->lsum[2][r] + ctl->lsum[3][r], tag);
     }
     tc_fence_before();
-    stamp_by(128, 9);
+    MASW_STAMP_BY(tr, 128, 9);
   }
 
   __syncthreads();
-  stamp(2);
+  MASW_STAMP(tr, 2);
+#ifdef MASW_TRACE
   if (tr && tid == 0) { tr[6] = ctl->plan[2]; unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); tr[7] = sm; }
+#endif
   if (ctl->error != 0) {
     if (tid == 0 && p.status) atomicOr(p.status, MASW_STATUS_WAIT_TIMEOUT);
   }
@@ -640,11 +646,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
   }
-  stamp(3);
+  MASW_STAMP(tr, 3);
   split_reduce_and_store<D, NQ, C::kThreads>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
   // the pool counter of the next launch (the other parity) is idle now: clear it
   if (split == 0 && tid == 0) p.tickets[(b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + ((ctl->plan[6] + 1) & 1)] = 0;
-  stamp(4);
+  MASW_STAMP(tr, 4);
 }
 
 }  // namespace masw

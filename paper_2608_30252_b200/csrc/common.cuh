@@ -1,6 +1,8 @@
 // Shared host/device helpers of the MASW library (sm_100a only).
 #pragma once
 
+#include <atomic>
+
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -16,7 +18,9 @@ namespace masw {
 void set_error(const char* fmt, ...);
 void count_launch(int n = 1);
 int check_cuda(cudaError_t e, const char* what);
-int sm_count();
+constexpr int kMaxDevices = 64;   // per-device caches (kernel attributes, SM counts, symbol addresses) are arrays of this size
+int current_device();             // index of the current CUDA device, clamped to [0, kMaxDevices)
+int sm_count();                   // SM count of the current device
 
 #define MASW_CUDA_TRY(expr)                                        \
   do {                                                             \
@@ -31,6 +35,19 @@ int sm_count();
       return (code);                                               \
     }                                                              \
   } while (0)
+
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute is per device, and a
+// process may drive several).  `once` is a static object of the launching function.
+struct PerDeviceOnce { std::atomic<bool> done[kMaxDevices]; };
+template <typename Kern>
+static inline int set_smem_once(Kern kern, int bytes, PerDeviceOnce& once) {
+  const int dev = current_device();
+  if (!once.done[dev].load(std::memory_order_acquire)) {
+    MASW_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    once.done[dev].store(true, std::memory_order_release);
+  }
+  return MASW_OK;
+}
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -99,14 +116,14 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t par
   return ok != 0;
 }
 
-// Bounded wait: gives up after kWaitLimit polls, so a lost copy can never hang the GPU.  Returns false on
-// give-up.  The first polls return at once (short waits stay cheap), later ones park the thread for up to
-// kParkNs each, which bounds the whole wait to a few seconds.
+// Bounded wait: gives up after `limit` polls (kWaitLimit unless the launch says otherwise), so a lost copy
+// can never hang the GPU.  Returns false on give-up.  The first poll returns at once (short waits stay
+// cheap), later ones park the thread for up to kParkNs each, which bounds the whole wait to a few seconds.
 constexpr int kWaitLimit = 1 << 20;
 constexpr uint32_t kParkNs = 4000;
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit = kWaitLimit) {
   if (mbar_try_wait(bar, parity)) return true;
-  for (int i = 0; i < kWaitLimit; ++i) {
+  for (int i = 0; i < limit; ++i) {
     if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
   }
   return false;
@@ -171,6 +188,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+
+// Phase stamps of the developer build (-DMASW_TRACE): thread `who` of the CTA writes %globaltimer into word
+// `slot` of the CTA's 16-word record.  The product build compiles them out.
+#ifdef MASW_TRACE
+#define MASW_STAMP_BY(tr, who, slot)                                              \
+  do {                                                                            \
+    if ((tr) != nullptr && threadIdx.x == (who)) {                                \
+      long long t_;                                                               \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_) : : "memory");         \
+      (tr)[slot] = t_;                                                            \
+    }                                                                             \
+  } while (0)
+#else
+#define MASW_STAMP_BY(tr, who, slot) do { } while (0)
+#endif
+#define MASW_STAMP(tr, slot) MASW_STAMP_BY(tr, 0, slot)
 
 #endif  // __CUDACC__
 

@@ -321,7 +321,10 @@ extern "C" int mem_get_state(masw_mem* mem, int32_t* t, int32_t* n_slots, int32_
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (t) MASW_CUDA_TRY(cudaMemcpyAsync(t, mem->d_t, sizeof(int) * B, cudaMemcpyDeviceToHost, st));
   if (n_slots) MASW_CUDA_TRY(cudaMemcpyAsync(n_slots, mem->d_slots, sizeof(int) * B, cudaMemcpyDeviceToHost, st));
-  if (status) MASW_CUDA_TRY(cudaMemcpyAsync(status, mem->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (status) {   // the bits accumulate between reads: a read returns them and starts over
+    MASW_CUDA_TRY(cudaMemcpyAsync(status, mem->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    MASW_CUDA_TRY(cudaMemsetAsync(mem->d_status, 0, sizeof(int), st));
+  }
   MASW_CUDA_TRY(cudaStreamSynchronize(st));
   return MASW_OK;
 }

@@ -132,9 +132,9 @@ def test_prefill_builds_the_memory_decoding_continues_from():
     g.close()
 
 
-@pytest.mark.parametrize("name", ["cfg3_8b_32k"])
+@pytest.mark.parametrize("name", ["cfg3_8b_32k", "cfg4_70b_32k"])
 def test_full_size_prefix_sampled_rows(name):
-    """The 32K prefix of the benchmark's draft shape, one layer: sampled rows (first and last tokens, rows
+    """The 32K prefix of the benchmark's draft shapes (head_dim 64 and head_dim 128), one layer: sampled rows (first and last tokens, rows
     around tile and window edges, slot rows) against the oracle, row by row."""
     wl = inputs.WORKLOADS[name]
     rng = inputs.rng_for(3, 0, 93)

@@ -36,6 +36,15 @@ def _case(rng, B, Hq, Hkv, D, P, T, cap=None, lens=None, q_scale=1.0, poison=Fal
     assert float(d.pow(2).mean().sqrt()) <= 2 * rel_tol * float(og.double().pow(2).mean().sqrt()) + 1e-12   # two noisy runs
     assert torch.allclose(lg, lg2, rtol=1e-3, atol=1e-3)
     oref, lref = oracle.verify_attend(f64(qb), f64(kb), f64(vb), lens)
+    # the deterministic mode (every tile assigned statically): same parity bar, and a repeat is bit-identical;
+    # its status word stays clear
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    od, ld = binding.verify_attend(k, v, kv_len, dev_bf16(qb), workspace=ws, deterministic=True, status=status)
+    od2, ld2 = binding.verify_attend(k, v, kv_len, dev_bf16(qb), workspace=ws, deterministic=True, status=status)
+    assert torch.equal(od, od2) and torch.equal(ld, ld2), "deterministic verify_attend is not run-to-run identical"
+    assert int(status.item()) == 0
+    assert_attention_close(od.cpu().numpy(), oref, ld.cpu().numpy(), lref, tag=f"deterministic verify B{B} Hq{Hq} T{T} P{P}",
+                           rel_tol=rel_tol)
     return assert_attention_close(og.cpu().numpy(), oref, lg.cpu().numpy(), lref, tag=f"verify B{B} Hq{Hq} T{T} P{P}", rel_tol=rel_tol)
 
 

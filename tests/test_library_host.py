@@ -86,6 +86,20 @@ def test_verify_and_accept_validate_before_launch(lib):
     assert rc == binding.MASW_EINVAL            # sampling without draft logits / uniforms
 
 
+def test_sampling_vocab_bound_and_no_developer_hooks_in_the_product_library(lib):
+    """temperature > 0 keeps 64-bit weight sums: a vocabulary of 2^17 or more is refused before any launch (greedy
+    has no such bound).  The product library exports none of the developer build's hooks."""
+    args = lambda V, temp: (C.c_void_p(0x1000), C.c_void_p(0x1100), C.c_void_p(0x2000), C.c_void_p(0x2100), 1, 4, V, temp,
+                            C.c_void_p(0x3000), C.c_void_p(0x4000), None)
+    assert lib.accept_reject(*args(131072, 1.0), C.c_void_p(0x5000), 16, None) == binding.MASW_EINVAL
+    assert "vocab" in lib.masw_last_error().decode()
+    assert lib.accept_reject(*args(131071, 1.0), C.c_void_p(0x5000), 16, None) == binding.MASW_ECAPACITY   # passes the bound, fails on the tiny workspace
+    assert lib.accept_reject(*args(200000, 0.0), C.c_void_p(0x5000), 16, None) == binding.MASW_ECAPACITY
+    assert lib.accept_reject_static(*args(131072, 1.0), None) == binding.MASW_EINVAL
+    for name in ("masw_debug_set_trace", "masw_debug_set_wait", "masw_debug_set_flags", "masw_debug_set_verify_legacy"):
+        assert not hasattr(lib, name), name
+
+
 def test_paged_verify_and_prefill_validate_before_launch(lib):
     """Bad arguments of the two newer entry points are refused on the host (fake pointers are never touched)."""
     vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t

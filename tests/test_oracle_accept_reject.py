@@ -6,7 +6,8 @@ import os
 import numpy as np
 
 import oracle
-from oracle.accept_reject import FRAC_BITS
+
+from oracle.accept_reject import FRAC_BITS, integer_weights
 from paper_2608_30252_b200 import inputs
 
 
@@ -128,6 +129,23 @@ def test_identical_distributions_always_accept_and_low_temperature_is_greedy():
     one_hot = np.full((1, 3, 50), -30.0); np.put_along_axis(one_hot, greedy_toks[..., None], 0.0, -1)
     n_s, out_s = oracle.accept_reject(tl, one_hot, greedy_toks, inputs.uniforms_24bit(rng, (1, 4)), 0.01)
     assert n_g[0] == n_s[0] == 3 and np.array_equal(out_g, out_s)
+
+
+def test_residual_weight_sum_fits_64_bits_below_vocab_2_pow_17():
+    """The sampler's largest sum: p and q flat on disjoint halves of the vocabulary give sum R = (V/2)^2 2^32 =
+    V^2 2^30 (every weight is 2^40, each residual 2^40 (V/2) 2^40 >> 48).  It reaches 2^64 exactly at V = 2^17,
+    which is why a 64-bit implementation must refuse V >= 131072 when sampling; V = 131070 still fits."""
+    for V, fits in ((131070, True), (131072, False)):
+        half = V // 2
+        lo, hi = -200.0, 0.0                                   # exp(-200) has integer weight 0
+        p = np.array([hi] * half + [lo] * (V - half))
+        q = np.array([lo] * half + [hi] * (V - half))
+        Ip, Iq = integer_weights(p, 1.0), integer_weights(q, 1.0)
+        assert Ip[0] == 1 << 40 and Ip[-1] == 0 and Iq[0] == 0 and Iq[-1] == 1 << 40
+        Zp, Zq = sum(Ip), sum(Iq)
+        total = sum(max(0, ip * Zq - iq * Zp) >> 48 for ip, iq in zip(Ip, Iq))
+        assert total == half * (V - half) << 32
+        assert (total < 1 << 64) == fits
 
 
 def test_eq1_reproduces_paper_tables(golden_dir):

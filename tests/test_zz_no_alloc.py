@@ -5,14 +5,15 @@ accept_reject_static serves callers that cannot allocate device memory where the
 decision is taken (all memory already handed to their own pool, or cudaMalloc ruled out because it
 would stall the device in the middle of decoding).  Its scratch is a fixed array inside the library,
 shared by every call on the device, so the test runs two calls back to back on different inputs and
-compares each with the workspace-taking entry point: the second call must not be disturbed by what
-the first one left behind."""
+compares each with the workspace-taking entry point and with the CPU oracle's decisions: the second
+call must not be disturbed by what the first one left behind."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_30252_b200 import binding, inputs
-from helpers import dev_bf16
+from helpers import dev_bf16, host_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -38,6 +39,11 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(temperature):
     assert int(status.item()) == 0
     for (n_ref, out_ref), (n, out) in zip(expected, got):
         assert torch.equal(n, n_ref) and torch.equal(out, out_ref)      # integer decisions: bit-exact
+    # and directly against the oracle's decisions on the same logits, tokens and uniforms
+    for (tl, dl, toks, u), (n, out) in zip(cases, got):
+        f = lambda t: oracle.bf16_bits_to_f64(host_bits(t))
+        n_ref, out_ref = oracle.accept_reject(f(tl), f(dl), toks.cpu().numpy(), u.cpu().numpy(), temperature)
+        assert np.array_equal(n.cpu().numpy(), n_ref) and np.array_equal(out.cpu().numpy(), out_ref)
     # and once more in the opposite order, so each shape also follows the other one
     again = [binding.accept_reject_static(tl, dl, toks, u, temperature) for tl, dl, toks, u in reversed(cases)]
     for (n_ref, out_ref), (n, out) in zip(reversed(expected), again):
