@@ -29,6 +29,7 @@ METRIC = "draft+verify attention us/step at 32K prefix"
 # summarised in profiles/attend_kernels_cfg2_full.md (34.22 MB measured for 33.575 MB of KV)
 NCU_TRAFFIC_RATIO = 34.03 / 33.575
 UNIT = "us/step"
+TRACE_WORDS = 32   # 64-bit words per CTA in the developer build's stamp records
 SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -257,6 +258,61 @@ def draft_comparators(wl, device, reps=20):
         mem.close()
         del mem
         torch.cuda.empty_cache()
+    return out
+
+
+def draft_launch_kinds(runner, reps=30):
+    """Microseconds per launch of each kind of draft launch, each timed as a CUDA graph of one pass over all draft
+    layers in the product library: `plain` = draft_append_attend following another layer's launch (the common
+    case: it runs ahead of its predecessor), `plain_after_counter_update` = the same with mem_advance(0) before
+    every launch (each launch then reads everything behind its wait, as the first layer of a draft step does),
+    `boundary` = draft_boundary_attend following another layer's launch."""
+    torch = runner.torch
+    wl, mem = runner.wl, runner.mem
+    q1, q2 = runner.view("dq0"), runner.view(f"dq{runner.slot_step}")
+    k, v = runner.view("dk0"), runner.view("dv0")
+
+    def plain():
+        for l in range(wl.d_layers):
+            mem.draft_append_attend(l, k[l], v[l], q1[l], out=runner.d_o1[l], lse=runner.d_lse1[l])
+
+    def plain_dirty():
+        for l in range(wl.d_layers):
+            mem.mem_advance(0)
+            mem.draft_append_attend(l, k[l], v[l], q1[l], out=runner.d_o1[l], lse=runner.d_lse1[l])
+
+    def advance_only():
+        for l in range(wl.d_layers):
+            mem.mem_advance(0)
+
+    def boundary():
+        for l in range(wl.d_layers):
+            mem.draft_boundary_attend(l, k[l], v[l], runner.view("hg")[l], runner.Wk[l], runner.Wv[l], runner.slot_pos, q2[l],
+                                      out=runner.d_o2[l], lse=runner.d_lse2[l])
+
+    out = {}
+    side = torch.cuda.Stream(device=runner.dev)
+    for name, fn in (("plain", plain), ("plain_after_counter_update", plain_dirty), ("counter_update_alone", advance_only),
+                     ("boundary", boundary)):
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            fn()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(3):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) * 1e3 / (reps * wl.d_layers)
+    out["plain_after_counter_update"] -= out.pop("counter_update_alone")
+    runner.mem.mem_rollback(runner.t_keep, runner.m_keep, slots_keep_max=wl.slots)
     return out
 
 
@@ -534,6 +590,7 @@ def run_gpu(args, wl):
         d_gbs = draft_bytes_step / (draft_us * 1e-6) / 1e9
         base = cpu_baseline(wl) if world == 1 and not args.no_cpu_baseline else None
         comp = None
+        kinds = draft_launch_kinds(runner) if world == 1 else None
         if world == 1:
             launches_per_step, in_bytes, out_bytes = runner.launches_per_step, runner.in_bytes, runner.out_bytes
             del runner
@@ -574,6 +631,8 @@ def run_gpu(args, wl):
             "clocks": clock_info,
             "device_status": status,
         }
+        if kinds is not None:
+            line["phases"]["draft_us_per_launch_by_kind"] = kinds
         if comp is not None:
             # the paper's comparison points for the draft side (Section 5.1, Table 3), same kernel, one launch per layer
             line["phases"]["draft_comparators_us_per_layer"] = {
@@ -749,7 +808,7 @@ def run_timeline(args, wl):
         r.draft_phase(); r.verify_phase(); r.tail_phase()
     torch.cuda.synchronize()
     n_cta_max = 160
-    buf = torch.zeros(n_cta_max * 16, dtype=torch.int64, device=dev)
+    buf = torch.zeros(n_cta_max * TRACE_WORDS, dtype=torch.int64, device=dev)
 
     def capture(fn, name, slots, reps=5):
         acc = []
@@ -760,7 +819,7 @@ def run_timeline(args, wl):
             fn()
             torch.cuda.synchronize()
             binding.debug_set_trace(None)
-            t = buf.cpu().numpy().reshape(-1, 16)
+            t = buf.cpu().numpy().reshape(-1, TRACE_WORDS)
             t = t[t[:, 4] > 0]
             t0 = t[:, 0].min()
             acc.append((t[:, [s_ for _, s_ in slots]] - t0) / 1000.0)
@@ -772,15 +831,68 @@ def run_timeline(args, wl):
                           "max": round(float(col.max(axis=1).mean()), 2)}
         print(json.dumps(row), flush=True)
 
+    def capture_chain(n_launch=6, reps=4):
+        """Consecutive draft layers replayed from one CUDA graph, one record area per launch: when each launch's
+        CTAs start, pass their wait, finish their tiles, publish and end, in microseconds from the first launch's
+        first CTA (what overlaps between dependent launches shows here, not in a single eager launch)."""
+        stride = n_cta_max * TRACE_WORDS
+        cbuf = torch.zeros(n_launch * stride, dtype=torch.int64, device=dev)
+        q, k, v = r.view("dq0"), r.view("dk0"), r.view("dv0")
+        layers = [l % wl.d_layers for l in range(n_launch)]
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            r.mem.mem_advance(0)                  # the first launch of the chain follows a counter update, as in a draft step
+            for l in layers:
+                r.mem.draft_append_attend(l, k[l], v[l], q[l], out=r.d_o1[l], lse=r.d_lse1[l])
+            torch.cuda.synchronize()
+            binding.debug_set_trace(cbuf, stride)
+            with torch.cuda.graph(g, stream=side):
+                r.mem.mem_advance(0)
+                for l in layers:
+                    r.mem.draft_append_attend(l, k[l], v[l], q[l], out=r.d_o1[l], lse=r.d_lse1[l])
+            binding.debug_set_trace(None)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(reps):
+            cbuf.zero_()
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            t = cbuf.cpu().numpy().reshape(n_launch, n_cta_max, TRACE_WORDS)
+            t0 = t[0][t[0][:, 4] > 0][:, 0].min()
+        ghz = 1.965   # SM clock under this load (cycle stamps -> microseconds)
+        for k_ in range(n_launch):
+            live = t[k_][t[k_][:, 4] > 0]
+            cols = (live[:, [0, 10, 4]] - t0) / 1000.0
+            row = {"chain_launch": k_, "layer": layers[k_], "ctas": int(live.shape[0]), "sms_used": int(len(set(live[:, 7].tolist()))),
+                   "unit": "us from the first launch's first CTA (last repetition): median (min-max)",
+                   **{name: f"{np.median(cols[:, c]):.2f} ({cols[:, c].min():.2f}-{cols[:, c].max():.2f})"
+                      for c, name in enumerate(["cta_start", "wait_passed", "end"])}}
+            # thread 0's cycle stamps, as microseconds after its wait passed
+            names = [("q_arrived", 2), ("warp0_tile_landed", 3), ("warp0_scores", 16), ("warp0_probabilities", 17), ("warp0_pv", 18),
+                     ("warp0_tile_done", 19), ("tiles_consumed", 8), ("partials_in_smem", 20), ("published", 9),
+                     ("first_item_complete", 11), ("all_items_complete", 12), ("combined", 21), ("outputs_stored", 22), ("end", 13)]
+            for name, slot in names:
+                ok_rows = live[live[:, slot] > 0]
+                if len(ok_rows):
+                    d = (ok_rows[:, slot] - ok_rows[:, 1]) / ghz / 1000.0
+                    row["after_wait_" + name] = f"{np.median(d):.2f} ({d.min():.2f}-{d.max():.2f})"
+            print(json.dumps(row), flush=True)
+
+    if wl.d_q_heads // wl.d_kv_heads <= 8:
+        capture_chain()
+
     L = min(3, wl.d_layers - 1)
     q1, q2 = r.view("dq0"), r.view(f"dq{r.slot_step}")
     k, v = r.view("dk0"), r.view("dv0")
     mma = [("cta_start", 0), ("prologue_done", 1), ("tiles_consumed", 2), ("partial_published", 3), ("end", 4)]
+    draft = [("cta_start", 0), ("wait_passed", 10), ("end", 4)]   # the draft kernel's inner phases are cycle stamps (chain rows above)
     capture(lambda: r.mem.draft_append_attend(L, k[L], v[L], q1[L], out=r.d_o1[L], lse=r.d_lse1[L]),
-            "draft_append_attend (attend_kernel)", mma)
+            "draft_append_attend (attend_draft_kernel)", draft)
     capture(lambda: r.mem.draft_boundary_attend(L, k[L], v[L], r.view("hg")[L], r.Wk[L], r.Wv[L], r.slot_pos, q2[L],
                                                 out=r.d_o2[L], lse=r.d_lse2[L]),
-            "draft_boundary_attend (attend_kernel + slot projection)", mma)
+            "draft_boundary_attend (attend_draft_kernel + slot projection)", draft)
     vq = r.view("vq")
     LT = min(5, wl.t_layers - 1)
     tc = [("cta_start", 0), ("softmax_loop_end", 8), ("partial_published", 9), ("before_reduce", 3), ("end", 4)]

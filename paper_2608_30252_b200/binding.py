@@ -433,10 +433,12 @@ def load_trace() -> C.CDLL:
     global _trace_lib
     if _trace_lib is None:
         lib = _open(TRACE_LIB_PATH)
-        lib.masw_debug_set_trace.argtypes = [C.c_void_p]
+        lib.masw_debug_set_trace.argtypes = [C.c_void_p, C.c_longlong]
         lib.masw_debug_set_trace.restype = None
         lib.masw_debug_set_wait.argtypes = [C.c_int, C.c_int]
         lib.masw_debug_set_wait.restype = None
+        lib.masw_debug_set_flags.argtypes = [C.c_int]
+        lib.masw_debug_set_flags.restype = None
         _trace_lib = lib
     return _trace_lib
 
@@ -447,14 +449,21 @@ def select_trace_build() -> None:
     _lib = load_trace()
 
 
-def debug_set_trace(buffer) -> None:
+def debug_set_trace(buffer, stride_words=0) -> None:
     """Developer build: while `buffer` (an int64 CUDA tensor of at least 16 words per CTA of the next launches)
-    is set, the attention kernels of libmasw_trace.so write a few %globaltimer stamps per CTA into it.  Pass
-    None to switch the stamps off again."""
-    load_trace().masw_debug_set_trace(C.c_void_p(buffer.data_ptr()) if buffer is not None else None)
+    is set, the attention kernels of libmasw_trace.so write a few %globaltimer stamps per CTA into it.  With
+    stride_words > 0 every later launch writes `stride_words` further into the buffer (a chain of launches, also
+    when captured into a CUDA graph, then keeps one record area per launch).  Pass None to switch the stamps off."""
+    load_trace().masw_debug_set_trace(C.c_void_p(buffer.data_ptr()) if buffer is not None else None, int(stride_words))
 
 
 def debug_set_wait(wait_limit=0, drop_tile=-1) -> None:
     """Developer build: polls after which the kernels' bounded waits give up (0 = the normal limit) and the
     CTA-local index of one tile whose copy is armed but never issued (-1 = none)."""
     load_trace().masw_debug_set_wait(int(wait_limit), int(drop_tile))
+
+
+def debug_set_flags(flags=0) -> None:
+    """Developer build, timing experiments on the draft kernel (results are then meaningless): 1 = no cross-split
+    reduction, 2 = no tile arithmetic, 4 = never ahead of the predecessor."""
+    load_trace().masw_debug_set_flags(int(flags))

@@ -3,6 +3,7 @@
 #include <mutex>
 #include <vector>
 
+#include "attend_draft_kernel.cuh"
 #include "attend_kernel.cuh"
 #include "attend_tc_kernel.cuh"
 #include "mem_handle.cuh"
@@ -14,9 +15,18 @@ namespace masw {
 // timestamps, a shortened limit for the kernels' bounded waits, and the index of one tile whose copy is left
 // out so that such a wait runs out (the way the give-up path is tested without any fault)
 static long long* g_trace = nullptr;
+static long long g_trace_stride = 0;   // words by which the record area advances from one launch to the next (0: all launches share it)
+static long long g_trace_launch = 0;
 static int g_wait_limit = kWaitLimit;
 static int g_drop_tile = -1;
-static void apply_debug(AttendParams& p) { p.trace = g_trace; p.wait_limit = g_wait_limit; p.drop_tile = g_drop_tile; }
+static int g_debug_flags = 0;
+static void apply_debug(AttendParams& p) {
+  p.debug_flags = g_debug_flags;
+  if (g_debug_flags & 4) p.early = 0;
+  p.trace = g_trace ? g_trace + (g_trace_launch++) * g_trace_stride : nullptr;
+  p.wait_limit = g_wait_limit;
+  p.drop_tile = g_drop_tile;
+}
 #else
 static void apply_debug(AttendParams&) {}
 #endif
@@ -29,6 +39,7 @@ static int launch_attend(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendP
   auto kern = attend_kernel<D, MT, EW, TE, NSTAGE, CT>;
   static PerDeviceOnce once;
   { const int rc = set_smem_once(kern, C::kSmemBytes, once); if (rc != MASW_OK) return rc; }
+  p.early = 0;
   int splits = (sm_count() * CT) / (B * Hkv);
   if (splits > splits_max) splits = splits_max;
   if (splits > tiles_upper) splits = tiles_upper;
@@ -48,6 +59,46 @@ static int launch_attend(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendP
   if (splits > 1) { attr[na].id = cudaLaunchAttributeCooperative; attr[na].val.cooperative = 1; ++na; }
   // the kernel may be set up while its predecessor in the stream drains: it touches no global memory before
   // its griddepcontrol.wait
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na;
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmK, tmV, p));
+  count_launch();
+  return MASW_OK;
+}
+
+// The draft's decode launch for up to eight query rows per KV head: one CTA per SM and launch, but a footprint
+// that lets the next layer's CTAs become resident beside this layer's (see attend_draft_kernel.cuh).
+template <int D>
+static int launch_attend_draft(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendParams p, int B, int Hkv,
+                               int tiles_upper, int splits_max, cudaStream_t st) {
+  using C = DraftCfg<D>;
+  auto kern = attend_draft_kernel<D>;
+  static PerDeviceOnce once;
+  {
+    const int dev = current_device();
+    if (!once.done[dev].load(std::memory_order_acquire)) {
+      // the whole configurable array as shared memory, so that two 113 KB CTAs fit on an SM
+      MASW_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+    }
+    const int rc = set_smem_once(kern, C::kSmemBytes, once);
+    if (rc != MASW_OK) return rc;
+  }
+  int splits = sm_count() / (B * Hkv);
+  if (splits > splits_max) splits = splits_max;
+  if (splits > tiles_upper) splits = tiles_upper;
+  if (splits < 1) splits = 1;
+  p.splits = splits;
+  p.wait_limit = kWaitLimit;
+  apply_debug(p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(splits, Hkv, B);
+  cfg.blockDim = dim3(C::kThreads, 1, 1);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (splits > 1) { attr[na].id = cudaLaunchAttributeCooperative; attr[na].val.cooperative = 1; ++na; }
   attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na;
   cfg.attrs = attr;
   cfg.numAttrs = na;
@@ -173,11 +224,16 @@ int get_kv_maps(const masw_kv_desc& kv, int box, CUtensorMap* tk, CUtensorMap* t
 using namespace masw;
 
 #ifdef MASW_TRACE
-extern "C" void masw_debug_set_trace(void* device_buffer) { g_trace = static_cast<long long*>(device_buffer); }
+extern "C" void masw_debug_set_trace(void* device_buffer, long long stride_words) {
+  g_trace = static_cast<long long*>(device_buffer);
+  g_trace_stride = stride_words;
+  g_trace_launch = 0;
+}
 extern "C" void masw_debug_set_wait(int wait_limit, int drop_tile) {
   g_wait_limit = wait_limit > 0 ? wait_limit : kWaitLimit;
   g_drop_tile = drop_tile;
 }
+extern "C" void masw_debug_set_flags(int flags) { g_debug_flags = flags; }
 #endif
 
 struct SlotInputs {
@@ -227,8 +283,23 @@ static int draft_attend_impl(masw_mem* mem, int layer, const void* k_raw, const 
   const bool te32 = (tile_entries(c.head_dim, mt) == 32);
   const CUtensorMap& tk = te32 ? mem->tmK32[layer] : mem->tmK64[layer];
   const CUtensorMap& tv = te32 ? mem->tmV32[layer] : mem->tmV64[layer];
-  return dispatch_attend(c.head_dim, mt, tk, tv, p, c.batch, c.n_kv_heads, entries_upper, 4, mem->L.splits_max,
+  int rc;
+  if (n_q * mem->G <= 8) {
+    // a slot row whose slot was written by mem_update (not by this launch) reads that entry: never ahead of the wait
+    p.early = (mem->kv_clean && !(last_row_is_slot && slot.h_g == nullptr)) ? 1 : 0;
+    const int te = (c.head_dim == 64) ? DraftCfg<64>::TE : DraftCfg<128>::TE;   // equals tile_entries(head_dim, 1): same tensor maps
+    const int tiles_upper = (entries_upper + te - 1) / te + 4;
+    rc = (c.head_dim == 64)
+             ? launch_attend_draft<64>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, static_cast<cudaStream_t>(stream))
+             : launch_attend_draft<128>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, static_cast<cudaStream_t>(stream));
+  } else {
+    rc = dispatch_attend(c.head_dim, mt, tk, tv, p, c.batch, c.n_kv_heads, entries_upper, 4, mem->L.splits_max,
                          static_cast<cudaStream_t>(stream));
+  }
+  // either kernel waits for its predecessor before it lets a successor start and writes neither the counters
+  // nor another layer's K/V: the next layer's launch may read those early
+  mem->kv_clean = (rc == MASW_OK);
+  return rc;
 }
 
 extern "C" int draft_attend(masw_mem* mem, int layer, const void* q, int n_q, int last_row_is_slot, float* o,

@@ -59,12 +59,16 @@ struct AttendParams {
   int max_pages;
   int splits;
   float scale_log2e;
-  int wait_limit;          // polls after which a bounded wait gives up (kWaitLimit in normal operation)
+  int wait_limit;          // polls after which a bounded wait gives up: read by the developer build only (MASW_WAIT_LIMIT)
+  int early;               // draft (attend_draft_kernel): the counters, slot_pos and this layer's K/V are not written by
+                           // the launch's immediate predecessor in the stream, so they may be read before the wait
   int deterministic;       // verify (tcgen05 kernel): every tile assigned statically, results repeat bit for bit
 #ifdef MASW_TRACE
   long long* trace;        // developer build: per-CTA phase timestamps (null = off)
   int drop_tile;           // developer build: the copy of this CTA-local tile is armed but never issued (-1 = off),
                            // which makes a bounded wait run out without any fault
+  int debug_flags;         // developer build, draft kernel: 1 = no cross-split reduction, 2 = no tile arithmetic,
+                           // 4 = never ahead of the predecessor (timing experiments; results are then meaningless)
 #endif
 };
 
@@ -164,7 +168,7 @@ __device__ __forceinline__ void rec_fetch_item(const unsigned long long* ml_rec,
 template <int D, int KROWS, int NTHREADS>
 __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, int b, int kvh, int split, int n_rows,
                                                        int epoch, float* scratch, int tid,
-                                                       const double* rope_cs = nullptr) {
+                                                       const double* rope_cs = nullptr, long long* tr = nullptr) {
   constexpr float kNegInf = -INFINITY;
   const int bh = b * p.Hkv + kvh;
   __syncthreads();
@@ -234,7 +238,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
               all_ok &= r0.ok && r1.ok;
             }
           }
-          for (int it = 0; !all_ok && it < p.wait_limit; ++it) {   // a split that has not published yet
+          for (int it = 0; !all_ok && it < MASW_WAIT_LIMIT(p); ++it) {   // a split that has not published yet
             __nanosleep(20);
             all_ok = true;
 #pragma unroll
@@ -336,7 +340,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
             all_ok &= okv[u];
           }
         }
-        for (int it = 0; !all_ok && it < p.wait_limit; ++it) {   // a split that has not published yet
+        for (int it = 0; !all_ok && it < MASW_WAIT_LIMIT(p); ++it) {   // a split that has not published yet
           __nanosleep(20);
           all_ok = true;
 #pragma unroll
@@ -350,6 +354,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
           }
         }
         timed_out |= !all_ok;
+        MASW_CLOCK(tr, 11);   // developer build: thread 0 holds every split's record of its first item
         float mb = m_run2;
 #pragma unroll
         for (int u = 0; u < 6; ++u) if (sp0 + u * kGroups < splits) mb = fmaxf(mb, ml[u].x);
@@ -371,6 +376,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
       dst[0] = m_run2; dst[1] = l_run2; dst[2] = o4.x; dst[3] = o4.y; dst[4] = o4.z; dst[5] = o4.w;
     }
     __syncthreads();
+    MASW_CLOCK(tr, 12);     // developer build: every item of this CTA has all its records
     if (live && grp == 0) {
       float2 part[kGroups][3];   // m, l | o.x, o.y | o.z, o.w of each group's partial
 #pragma unroll
@@ -395,12 +401,14 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
         l += w_new;
         o.x += w_new * v_new.x; o.y += w_new * v_new.y; o.z += w_new * v_new.z; o.w += w_new * v_new.w;
       }
+      MASW_CLOCK(tr, 21);     // developer build: combined, before the stores
       const float inv = (l > 0.f) ? __frcp_rn(l) : 0.f;
       o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
       *reinterpret_cast<float4*>(out_o) = o;
       if (out_bf16) *reinterpret_cast<uint2*>(out_bf16) = make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
       if (out_lse) *out_lse = (l > 0.f) ? (m + __log2f(l)) * 0.6931471805599453f : kNegInf;
     }
+    MASW_CLOCK(tr, 22);     // developer build: this CTA's outputs are stored
     __syncthreads();
   }
   if (timed_out && p.status) atomicOr(p.status, MASW_STATUS_WAIT_TIMEOUT);
@@ -466,7 +474,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   const int n_rows = p.n_q * p.G;  // real query rows of this KV head
 
 #ifdef MASW_TRACE
-  long long* tr = p.trace ? p.trace + (static_cast<size_t>((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)) * 16 : nullptr;
+  long long* tr = p.trace ? p.trace + (static_cast<size_t>((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)) * kTraceWords : nullptr;
 #endif
   MASW_STAMP(tr, 0);
   const bool is_producer = (tid == C::kConsumerWarps * 32);   // lane 0 of the producer warp
@@ -625,7 +633,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         const int row0 = plan[8 + 4 * seg] + i0;
         const int stage = i % NSTAGE;
         const int round = i / NSTAGE;
-        ok = mbar_wait_bounded(&empty_bar[stage], (round - 1) & 1, p.wait_limit);
+        ok = mbar_wait_bounded(&empty_bar[stage], (round - 1) & 1, MASW_WAIT_LIMIT(p));
         if (!ok) break;
         uint8_t* kdst = pipe + stage * C::kStageBytes;
         uint8_t* vdst = kdst + C::kTileBytes;
@@ -732,7 +740,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
       }
 
-      ok = mbar_wait_bounded(&full_bar[stage], parity, p.wait_limit);
+      ok = mbar_wait_bounded(&full_bar[stage], parity, MASW_WAIT_LIMIT(p));
       if (!ok) break;
 
       uint8_t* ksm = pipe + stage * C::kStageBytes;
@@ -935,7 +943,7 @@ attend_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     if (tid == 0) {
       const int issued = plan[5];
       for (int i = max(0, issued - NSTAGE); i < issued; ++i) {
-        mbar_wait_bounded(&full_bar[i % NSTAGE], (i / NSTAGE) & 1, p.wait_limit);
+        mbar_wait_bounded(&full_bar[i % NSTAGE], (i / NSTAGE) & 1, MASW_WAIT_LIMIT(p));
       }
     }
     __syncthreads();

@@ -188,7 +188,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const int n_rows = p.n_q * p.G;
 
 #ifdef MASW_TRACE
-  long long* tr = p.trace ? p.trace + (static_cast<size_t>((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)) * 16 : nullptr;
+  long long* tr = p.trace ? p.trace + (static_cast<size_t>((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x)) * kTraceWords : nullptr;
 #endif
   MASW_STAMP(tr, 0);
   // producer state (thread 0 only): the schedule and the pool claim in flight
@@ -334,7 +334,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       int ik = n_early, iv = n_early;   // the first tiles were issued in the prologue
       bool k_done = false, v_done = false;
       int idle = 0;
-      while ((!k_done || !v_done) && idle < p.wait_limit) {
+      while ((!k_done || !v_done) && idle < MASW_WAIT_LIMIT(p)) {
         bool progressed = false;
         if (!k_done && (ik < NK || mbar_try_wait(&ctl->k_empty[ik % NK], (ik / NK - 1) & 1))) {
           const int id = resolve(ik);
@@ -392,8 +392,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       for (int i = 0; ok; ++i) {
         {
           const int sb = i & 1;
-          ok = mbar_wait_bounded(&ctl->k_full[i % NK], (i / NK) & 1, p.wait_limit);
-          if (ok && i >= 2) ok = mbar_wait_bounded(&ctl->s_empty[sb], ((i >> 1) - 1) & 1, p.wait_limit);
+          ok = mbar_wait_bounded(&ctl->k_full[i % NK], (i / NK) & 1, MASW_WAIT_LIMIT(p));
+          if (ok && i >= 2) ok = mbar_wait_bounded(&ctl->s_empty[sb], ((i >> 1) - 1) & 1, MASW_WAIT_LIMIT(p));
           if (!ok) break;
           if (ctl->tile_id[i & 15] < 0) {
             n_end = i;
@@ -413,8 +413,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         if (i >= 1) {
           const int j = i - 1;
-          ok = mbar_wait_bounded(&ctl->p_full[j & 1], (j >> 1) & 1, p.wait_limit);
-          if (ok) ok = mbar_wait_bounded(&ctl->v_full[j % NV], (j / NV) & 1, p.wait_limit);
+          ok = mbar_wait_bounded(&ctl->p_full[j & 1], (j >> 1) & 1, MASW_WAIT_LIMIT(p));
+          if (ok) ok = mbar_wait_bounded(&ctl->v_full[j % NV], (j / NV) & 1, MASW_WAIT_LIMIT(p));
           if (!ok) break;
           tc_fence_after();
           const uint32_t v_base = smem_u32(v_ring + (j % NV) * C::kTileBytes);
@@ -458,7 +458,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     volatile int* stop = &ctl->stop[grp];
     for (int i = 0;; ++i) {
       const int sb = i & 1;
-      if (ok) ok = mbar_wait_bounded(&ctl->s_full[sb], (i >> 1) & 1, p.wait_limit);
+      if (ok) ok = mbar_wait_bounded(&ctl->s_full[sb], (i >> 1) & 1, MASW_WAIT_LIMIT(p));
       ok = __all_sync(0xffffffffu, ok);
       const int tile = ctl->tile_id[i & 15];
       // The loop ends for the whole group at the named barrier below: at the end-of-stream marker, or
@@ -542,9 +542,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
       // the P tile is double-buffered: tile i - 2's P.V must be complete before its buffer is reused;
       // only a moved maximum has to wait for tile i - 1's P.V, to rescale O^T in tensor memory
-      if (i >= 2 && ok) ok = mbar_wait_bounded(&ctl->p_empty[i & 1], ((i >> 1) - 1) & 1, p.wait_limit);
+      if (i >= 2 && ok) ok = mbar_wait_bounded(&ctl->p_empty[i & 1], ((i >> 1) - 1) & 1, MASW_WAIT_LIMIT(p));
       if (i > 0 && any_changed) {
-        if (ok) ok = mbar_wait_bounded(&ctl->o_ready, (i - 1) & 1, p.wait_limit);
+        if (ok) ok = mbar_wait_bounded(&ctl->o_ready, (i - 1) & 1, MASW_WAIT_LIMIT(p));
         ok = __all_sync(0xffffffffu, ok);   // the tensor-memory accesses below are warp-wide
         tc_fence_after();
         if (ok) {
@@ -574,7 +574,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       // entries beyond the cache length hold foreign bytes: zero their V rows (their probability is 0,
       // but 0 x non-finite would poison the accumulator); the first group does it
       if (grp == 0 && (tile + 1) * C::kTile > kv_total) {   // only the last tile of the cache can have such rows
-        if (ok) ok = mbar_wait_bounded(&ctl->v_full[i % NV], (i / NV) & 1, p.wait_limit);   // the tile must have landed before it is patched
+        if (ok) ok = mbar_wait_bounded(&ctl->v_full[i % NV], (i / NV) & 1, MASW_WAIT_LIMIT(p));   // the tile must have landed before it is patched
         // rows [valid, 128) are one contiguous range in each 64-column half of the tile (the swizzle
         // permutes inside a row group, and whole rows are cleared); consecutive threads clear
         // consecutive 16-byte chunks, which is free of bank conflicts
@@ -599,7 +599,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int tag = ctl->plan[6] + 1;   // this launch's epoch tag
     bool have_o = ok && n_tiles > 0;
     if (have_o) {
-      have_o = mbar_wait_bounded(&ctl->o_ready, (n_tiles - 1) & 1, p.wait_limit);
+      have_o = mbar_wait_bounded(&ctl->o_ready, (n_tiles - 1) & 1, MASW_WAIT_LIMIT(p));
       tc_fence_after();
     }
     have_o = __all_sync(0xffffffffu, have_o);

@@ -170,6 +170,19 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, ui
                : "r"(addr));
 }
 
+__device__ __forceinline__ void ldmatrix_x2(uint32_t& r0, uint32_t& r1, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+
+// A hint that brings one line into L2; no value is read, so it may name memory another kernel is still writing.
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
 // D += A(16x16, row) * B(16x8, col), bf16 inputs, fp32 accumulate.
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -189,8 +202,18 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// The limit of the kernels' bounded waits: a launch parameter in the developer build (a test shortens it to make a
+// wait run out), the compile-time constant in the product build (the polling loops compile tighter with it).
+#ifdef MASW_TRACE
+#define MASW_WAIT_LIMIT(p) ((p).wait_limit)
+#else
+#define MASW_WAIT_LIMIT(p) (::masw::kWaitLimit)
+#endif
+
+constexpr int kTraceWords = 32;   // developer build: 64-bit words of one CTA's stamp record
+
 // Phase stamps of the developer build (-DMASW_TRACE): thread `who` of the CTA writes %globaltimer into word
-// `slot` of the CTA's 16-word record.  The product build compiles them out.
+// `slot` of the CTA's record.  The product build compiles them out.
 #ifdef MASW_TRACE
 #define MASW_STAMP_BY(tr, who, slot)                                              \
   do {                                                                            \
@@ -204,6 +227,15 @@ __device__ __forceinline__ float fast_exp2(float x) {
 #define MASW_STAMP_BY(tr, who, slot) do { } while (0)
 #endif
 #define MASW_STAMP(tr, slot) MASW_STAMP_BY(tr, 0, slot)
+// The SM's cycle counter instead (cheap to read, comparable only inside one CTA): thread 0 of the CTA.
+#ifdef MASW_TRACE
+#define MASW_CLOCK(tr, slot)                                                      \
+  do {                                                                            \
+    if ((tr) != nullptr && threadIdx.x == 0) (tr)[slot] = clock64();              \
+  } while (0)
+#else
+#define MASW_CLOCK(tr, slot) do { } while (0)
+#endif
 
 #endif  // __CUDACC__
 

@@ -268,6 +268,7 @@ extern "C" void mem_free(masw_mem* mem) { delete mem; }
 extern "C" int mem_load(masw_mem* mem, int layer, int region, const void* k, const void* v, int first, int n,
                         const int64_t strides[3], void* stream) {
   MASW_REQUIRE(mem != nullptr && k != nullptr && v != nullptr && strides != nullptr, MASW_EINVAL, "mem_load: null argument");
+  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   MASW_REQUIRE(layer >= 0 && layer < mem->cfg.n_layers, MASW_EINVAL, "mem_load: layer %d out of range", layer);
   MASW_REQUIRE(n >= 0 && first >= 0, MASW_EINVAL, "mem_load: negative count or index");
   MASW_REQUIRE(aligned16(k) && aligned16(v), MASW_EALIGN, "mem_load: pointers must be 16-byte aligned");
@@ -296,6 +297,7 @@ extern "C" int mem_load(masw_mem* mem, int layer, int region, const void* k, con
 
 extern "C" int mem_set_state(masw_mem* mem, const int32_t* t, const int32_t* n_slots, void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_set_state: null handle");
+  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   const int B = mem->cfg.batch;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (t) {
@@ -333,6 +335,7 @@ extern "C" int mem_update(masw_mem* mem, int layer, const void* k_raw, const voi
                           const void* Wk_g, const void* Wv_g, const int32_t* slot_pos, const uint8_t* active,
                           void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_update: null handle");
+  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   MASW_REQUIRE(layer >= 0 && layer < mem->cfg.n_layers, MASW_EINVAL, "mem_update: layer %d out of range", layer);
   const masw_config& c = mem->cfg;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -379,6 +382,7 @@ extern "C" int mem_update(masw_mem* mem, int layer, const void* k_raw, const voi
 
 extern "C" int mem_advance(masw_mem* mem, int n_tokens, int add_slot, const uint8_t* active, void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_advance: null handle");
+  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   MASW_REQUIRE(n_tokens >= 0 && n_tokens <= mem->cfg.gamma_max, MASW_EINVAL, "mem_advance: n_tokens %d outside [0, gamma_max]", n_tokens);
   if (add_slot) {
     MASW_REQUIRE(mem->slots_upper < mem->cfg.max_slots, MASW_ECAPACITY, "mem_advance: slot region full");
@@ -395,6 +399,7 @@ extern "C" int mem_advance(masw_mem* mem, int n_tokens, int add_slot, const uint
 extern "C" int mem_rollback(masw_mem* mem, const int32_t* t_keep, const int32_t* slots_keep, int slots_keep_max,
                             void* stream) {
   MASW_REQUIRE(mem != nullptr && t_keep != nullptr && slots_keep != nullptr, MASW_EINVAL, "mem_rollback: null argument");
+  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   if (slots_keep_max >= 0) mem->slots_upper = std::min(mem->slots_upper, slots_keep_max);
   const int B = mem->cfg.batch;
   rollback_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(mem->d_t, mem->d_slots, t_keep, slots_keep, B);

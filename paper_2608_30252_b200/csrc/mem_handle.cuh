@@ -77,6 +77,12 @@ struct masw_mem {
   unsigned long long* d_part_slot;
   std::vector<CUtensorMap> tmK32, tmV32, tmK64, tmV64;  // per layer, box of 32 / 64 entries
   int slots_upper;  // host-side upper bound on any sequence's committed slot count
+  // True while the last call on this handle was a draft attention launch: such a launch waits for its
+  // predecessor before it lets its successor start, and writes neither the counters nor another layer's K/V,
+  // so the next layer's launch may read those ahead of its own wait.  Every call that writes the counters
+  // or the arena through another path (mem_update, mem_load, mem_advance, mem_rollback, mem_set_state, the
+  // prefill import) clears it.
+  bool kv_clean = false;
 
   __nv_bfloat16* k_layer(int layer) const {
     return reinterpret_cast<__nv_bfloat16*>(arena) + static_cast<size_t>(layer) * 2 * tensor_elems;

@@ -205,14 +205,20 @@ def _loaded_case(wl, layer_count, layer, rng, fused=False):
     g.mem_set_state(t=[t0] * B, n_slots=[M] * B)
     kn, vn = inputs.normal_bf16(rng, (B, 1, Hkv, D)), inputs.normal_bf16(rng, (B, 1, Hkv, D))
     q = inputs.normal_bf16(rng, (B, 1, Hq, D))
+    # The first launch follows a counter update and reads everything behind its wait; the launches after it
+    # follow an attention launch and may run ahead of it (plan and K/V copies before the wait, the CTA's first
+    # tile kept in registers).  The two orders sum the same entries in a different order, so each is checked
+    # against the oracle, and the repeated order must give the same bits (run-to-run determinism).
     if fused:      # the launch the benchmark times: append fused into the attention
-        og, lg = g.draft_append_attend(layer, dev_bf16(kn), dev_bf16(vn), dev_bf16(q))
-        og2, lg2 = g.draft_append_attend(layer, dev_bf16(kn), dev_bf16(vn), dev_bf16(q))
+        call = lambda: g.draft_append_attend(layer, dev_bf16(kn), dev_bf16(vn), dev_bf16(q))
     else:
         g.mem_update(layer, k_raw=dev_bf16(kn), v_raw=dev_bf16(vn))
-        og, lg = g.draft_attend(layer, dev_bf16(q))
-        og2, lg2 = g.draft_attend(layer, dev_bf16(q))
-    assert torch.equal(og, og2) and torch.equal(lg, lg2)          # run-to-run bitwise determinism
+        call = lambda: g.draft_attend(layer, dev_bf16(q))
+    (og, lg), (og2, lg2), (og3, lg3) = call(), call(), call()
+    assert torch.equal(og2, og3) and torch.equal(lg2, lg3)
+    g.mem_advance(0)                                              # a counter update: the next launch waits first again
+    og4, lg4 = call()
+    assert torch.equal(og, og4) and torch.equal(lg, lg4)
     # oracle: the plain definition over the explicit entry list
     G = Hq // Hkv
     scale = 1 / math.sqrt(D)
@@ -226,6 +232,7 @@ def _loaded_case(wl, layer_count, layer, rng, fused=False):
         assert len(K) == S + M + W
         for h in range(Hq):
             oref[b, 0, h], lref[b, 0, h], _ = oracle.attend(f64(q[b, 0, h]), K[:, h // G], V[:, h // G], scale)
+    assert_attention_close(og2.cpu().numpy(), oref, lg2.cpu().numpy(), lref, tag=wl.name + " (ahead of its predecessor)", rel_tol=2e-4)
     mx, rel = assert_attention_close(og.cpu().numpy(), oref, lg.cpu().numpy(), lref, tag=wl.name, rel_tol=2e-4)
     assert g.mem_get_state()[2] == 0
     return mx, rel
