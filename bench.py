@@ -831,27 +831,35 @@ def run_timeline(args, wl):
                           "max": round(float(col.max(axis=1).mean()), 2)}
         print(json.dumps(row), flush=True)
 
-    def capture_chain(n_launch=6, reps=4):
+    def capture_chain(n_launch=6, reps=4, boundary=False):
         """Consecutive draft layers replayed from one CUDA graph, one record area per launch: when each launch's
         CTAs start, pass their wait, finish their tiles, publish and end, in microseconds from the first launch's
         first CTA (what overlaps between dependent launches shows here, not in a single eager launch)."""
         stride = n_cta_max * TRACE_WORDS
         cbuf = torch.zeros(n_launch * stride, dtype=torch.int64, device=dev)
-        q, k, v = r.view("dq0"), r.view("dk0"), r.view("dv0")
+        q, k, v = r.view(f"dq{r.slot_step}" if boundary else "dq0"), r.view("dk0"), r.view("dv0")
         layers = [l % wl.d_layers for l in range(n_launch)]
+
+        def launch(l):
+            if boundary:
+                r.mem.draft_boundary_attend(l, k[l], v[l], r.view("hg")[l], r.Wk[l], r.Wv[l], r.slot_pos, q[l],
+                                            out=r.d_o2[l], lse=r.d_lse2[l])
+            else:
+                r.mem.draft_append_attend(l, k[l], v[l], q[l], out=r.d_o1[l], lse=r.d_lse1[l])
+
         side = torch.cuda.Stream(device=dev)
         side.wait_stream(torch.cuda.current_stream())
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
             r.mem.mem_advance(0)                  # the first launch of the chain follows a counter update, as in a draft step
             for l in layers:
-                r.mem.draft_append_attend(l, k[l], v[l], q[l], out=r.d_o1[l], lse=r.d_lse1[l])
+                launch(l)
             torch.cuda.synchronize()
             binding.debug_set_trace(cbuf, stride)
             with torch.cuda.graph(g, stream=side):
                 r.mem.mem_advance(0)
                 for l in layers:
-                    r.mem.draft_append_attend(l, k[l], v[l], q[l], out=r.d_o1[l], lse=r.d_lse1[l])
+                    launch(l)
             binding.debug_set_trace(None)
         torch.cuda.current_stream().wait_stream(side)
         for _ in range(reps):
@@ -865,23 +873,29 @@ def run_timeline(args, wl):
         for k_ in range(n_launch):
             live = t[k_][t[k_][:, 4] > 0]
             cols = (live[:, [0, 10, 4]] - t0) / 1000.0
-            row = {"chain_launch": k_, "layer": layers[k_], "ctas": int(live.shape[0]), "sms_used": int(len(set(live[:, 7].tolist()))),
+            row = {"chain_launch": k_, "kind": "boundary" if boundary else "plain", "layer": layers[k_], "ctas": int(live.shape[0]), "sms_used": int(len(set(live[:, 7].tolist()))),
                    "unit": "us from the first launch's first CTA (last repetition): median (min-max)",
                    **{name: f"{np.median(cols[:, c]):.2f} ({cols[:, c].min():.2f}-{cols[:, c].max():.2f})"
                       for c, name in enumerate(["cta_start", "wait_passed", "end"])}}
             # thread 0's cycle stamps, as microseconds after its wait passed
-            names = [("q_arrived", 2), ("warp0_tile_landed", 3), ("warp0_scores", 16), ("warp0_probabilities", 17), ("warp0_pv", 18),
+            names = [("projection_loads_issued", 23), ("projection_summed", 24), ("q_arrived", 2), ("warp0_tile_landed", 3), ("warp0_scores", 16), ("warp0_probabilities", 17), ("warp0_pv", 18),
                      ("warp0_tile_done", 19), ("tiles_consumed", 8), ("partials_in_smem", 20), ("published", 9),
+                     ("reduction_starts", 26), ("slot_records_first_answer", 29), ("slot_records_summed", 25), ("slot_final", 27), ("slot_phase_over", 28),
                      ("first_item_complete", 11), ("all_items_complete", 12), ("combined", 21), ("outputs_stored", 22), ("end", 13)]
             for name, slot in names:
                 ok_rows = live[live[:, slot] > 0]
                 if len(ok_rows):
                     d = (ok_rows[:, slot] - ok_rows[:, 1]) / ghz / 1000.0
                     row["after_wait_" + name] = f"{np.median(d):.2f} ({d.min():.2f}-{d.max():.2f})"
+            if boundary:
+                flags = live[:, 30]
+                row["slot_records_all_there_at_first_load"] = f"{int((flags == 1).sum())} of {int((flags > 0).sum())} CTAs"
             print(json.dumps(row), flush=True)
 
     if wl.d_q_heads // wl.d_kv_heads <= 8:
         capture_chain()
+    if 2 * (wl.d_q_heads // wl.d_kv_heads) <= 8:
+        capture_chain(boundary=True)
 
     L = min(3, wl.d_layers - 1)
     q1, q2 = r.view("dq0"), r.view(f"dq{r.slot_step}")

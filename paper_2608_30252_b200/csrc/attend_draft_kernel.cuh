@@ -44,22 +44,21 @@ struct DraftCfg {
   // scratch that reuses the stages once every tile is consumed
   static constexpr int kMergeOff = 0;                                        // [kWarps][kRows][kMergeStride] + [kWarps][kRows][2]
   static constexpr int kMergeBytes = kWarps * kRows * (kMergeStride + 2) * 4;
-  static constexpr int kProjHsOff = 40 * 1024;                               // slot projection: hidden-state slice (<= 16 KB)
-  static constexpr int kProjRedOff = 56 * 1024;                              // [row lanes][2 D] partial sums (<= 18 KB)
-  static constexpr int kRopeOff = 80 * 1024;                                 // [D/2][2] doubles
   static constexpr int kReduceOff = 84 * 1024;                               // scratch of split_reduce_and_store
   static_assert(D == 64 || D == 128, "head_dim");
-  static_assert(kMergeBytes <= kProjHsOff, "merge scratch overlaps the projection staging");
-  static_assert(kReduceOff + kThreads * 24 + 8 * D + 64 <= kPipeBytes, "reduction scratch must fit in the stages");
+  static_assert(kMergeBytes <= kReduceOff, "merge scratch overlaps the reduction scratch");
+  static_assert(kReduceOff + 9216 + 24 * D <= kPipeBytes, "reduction scratch must fit in the stages");
+  static_assert(kThreads == 256, "draft_reduce_and_store is written for 256 threads");
   static_assert(kSmemBytes <= 113 * 1024, "two CTAs per SM");
 };
 
 struct DraftCtrl {
   uint64_t full_bar[8];
-  int plan[48];        // [0] nseg, [1] tile_begin, [2] tile_end, [3] error flag, [6] reduction epoch, [7] committed tokens t,
+  int plan[40];        // [0] nseg, [1] tile_begin, [2] tile_end, [3] error flag, [6] reduction epoch, [7] committed tokens t,
                        // [8 + 4 s ..] phys, len, xbase, kind of segment s, [32 + s] first tile of segment s (s = 0..nseg)
   int row_lo[kMaxSeg * 8], row_hi[kMaxSeg * 8];
   int armed[8];        // per stage: 1 + the CTA-local index of the tile the stage was last armed (and requested) for
+  float rope[128];     // boundary step: (cos, sin) of the new slot's D / 2 rotation angles (angles formed in double)
 };
 static_assert(sizeof(DraftCtrl) <= 1024, "control block");
 
@@ -76,6 +75,256 @@ __device__ __forceinline__ int ld_acquire_shared(const int* p) {
 }
 __device__ __forceinline__ void st_release_shared(int* p, int v) {
   asm volatile("st.release.cta.shared.b32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+
+
+// Cross-split reduction of the draft launch: split_reduce_and_store's scheme (tagged 64-bit records, every CTA
+// merges its slice of the (row, 4-column) items out of all splits' records in a fixed order) for eight rows and
+// 256 threads, with the boundary step's slot work moved ahead of the rendezvous.  The splits' partial sums of
+// K_g | V_g were published at the start of the launch, so they are here long before the attention partials:
+// the CTAs that need the new slot (split 0 stores it; the owners of slot-row items attend to it) sum them in
+// split order, rotate the key, round both to bf16 as stored and take the slot rows' scores against it while the
+// other splits are still publishing; behind the rendezvous only the final combine is left.
+// Must be called by all 256 threads; `scratch` is shared memory of at least 9 KB + 24 D bytes.
+template <int D>
+__device__ __forceinline__ void draft_reduce_and_store(const AttendParams& p, int b, int kvh, int split, int n_rows, int epoch,
+                                                       float* scratch, int tid, const float* rope_cs, long long* tr) {
+  constexpr float kNegInf = -INFINITY;
+  constexpr int NT = 256, KROWS = 8;
+  constexpr int kGroups = 8, kSlots = NT / kGroups;   // thread groups per item, items per batch
+  constexpr int kFetch = 3;   // splits whose records a group thread has in flight: 24 splits per round trip
+  const int bh = b * p.Hkv + kvh;
+  const int tag = epoch + 1;
+  const unsigned long long* all_o = p.part_o + static_cast<size_t>(bh) * p.splits * KROWS * D;
+  const unsigned long long* all_ml = p.part_ml + static_cast<size_t>(bh) * p.splits * KROWS * 2;
+  const int splits = p.splits;
+  const int n_items = n_rows * (D / 4);
+  const int per = (n_items + splits - 1) / splits;
+  const int i_begin = split * per;
+  const int my_items = max(0, min(n_items, i_begin + per) - i_begin);
+  float* gsm = scratch;                        // [kGroups][kSlots][6]: m, l, o4
+  float* psum = gsm + kGroups * kSlots * 6;    // [NT / D][2 D] partial sums of K_g | V_g
+  float* kg = psum + 2 * NT;                   // [D] key of the new slot (bf16 values); vg follows it
+  float* vg = kg + D;
+  float* sg = vg + D;                          // [G] scaled scores of the slot rows against it (log2 domain)
+  bool timed_out = false;
+  __syncthreads();   // the scratch is free
+
+  // ---- boundary step: what the slot phase needs is requested now and used behind the rendezvous of the
+  // attention partials (the splits published their sums of K_g | V_g at the start of the launch, so these
+  // records have long arrived; the loads ride along with the wait for the other splits' partials)
+  const int first_slot_item = (n_rows - p.G) * (D / 4);
+  const bool slot_term = p.h_g != nullptr && (p.active == nullptr || p.active[b] != 0) &&
+                         (split == 0 || i_begin + my_items > first_slot_item);
+  constexpr int kColGroups = NT / D;                        // thread (columns 2 c, 2 c + 1 of K | V, group): splits group, group + groups, ...
+  constexpr int kBatch = (D == 64) ? 5 : 10;                // 16-byte record pairs in flight per thread: up to 20 splits in one round trip
+  constexpr int kQPerLane = D / 32;
+  const unsigned long long* ps = p.part_slot + static_cast<size_t>(bh) * splits * 2 * D;
+  const int col = 2 * (tid % D), cgp = tid / D;
+  const int warp = tid >> 5, lane = tid & 31;
+  unsigned short qraw[kQPerLane];   // the slot rows' query values (warp g holds row g), converted when used
+  MASW_CLOCK(tr, 26);     // developer build: the reduction starts
+  if (slot_term) {
+#pragma unroll
+    for (int e = 0; e < kQPerLane; ++e) {
+      qraw[e] = 0;
+      if (warp < p.G)
+        qraw[e] = __ldg(reinterpret_cast<const unsigned short*>(p.q) +
+                        ((static_cast<size_t>(b) * p.n_q + (p.n_q - 1)) * p.Hq + kvh * p.G + warp) * D + lane + 32 * e);
+    }
+    // the splits' sums of this thread's column, in split order; the total goes to shared memory at once, so that
+    // nothing is held in registers while the attention partials are awaited
+    float sum = 0.f, sum_b = 0.f;
+    for (int sp0 = cgp; sp0 < splits; sp0 += kColGroups * kBatch) {
+      float sv[kBatch], sw[kBatch];
+      bool sok[kBatch];
+      bool all_ok = true;
+#pragma unroll
+      for (int e = 0; e < kBatch; ++e) {
+        sv[e] = 0.f; sw[e] = 0.f; sok[e] = true;
+        const int sp = sp0 + e * kColGroups;
+        if (sp < splits) {
+          const Rec2 r = rec_load2(ps + static_cast<size_t>(sp) * 2 * D + col, tag);
+          sv[e] = r.a; sw[e] = r.b; sok[e] = r.ok; all_ok &= r.ok;
+        }
+      }
+#ifdef MASW_TRACE
+      if (tr != nullptr && tid == 0) { tr[29] = clock64(); tr[30] = all_ok ? 1 : 2; }   // first answers are in; were they all there?
+#endif
+      for (int it = 0; !all_ok && it < MASW_WAIT_LIMIT(p); ++it) {   // a split that has not published yet
+        __nanosleep(20);
+        all_ok = true;
+#pragma unroll
+        for (int e = 0; e < kBatch; ++e) {
+          if (!sok[e]) {
+            const Rec2 r = rec_load2(ps + static_cast<size_t>(sp0 + e * kColGroups) * 2 * D + col, tag);
+            sv[e] = r.a; sw[e] = r.b; sok[e] = r.ok; all_ok &= r.ok;
+          }
+        }
+      }
+      timed_out |= !all_ok;
+#pragma unroll
+      for (int e = 0; e < kBatch; ++e) { sum += sv[e]; sum_b += sw[e]; }
+    }
+    psum[cgp * 2 * D + col] = sum;
+    psum[cgp * 2 * D + col + 1] = sum_b;
+    MASW_CLOCK(tr, 25);   // developer build: this thread's slot records are summed
+  }
+  // The rest of the slot phase; called by the whole CTA once the first batch of items has its records (a
+  // __syncthreads() lies between the sums above and this).
+  auto slot_phase = [&]() {
+    // unit u < D / 2: key columns (u, u + D / 2), rotated together; unit D / 2 + j: value columns (2 j, 2 j + 1)
+    if (tid < D) {
+      const int u = tid;
+      const bool is_k = u < D / 2;
+      const int c0 = is_k ? u : D + 2 * (u - D / 2);
+      const int c1 = is_k ? u + D / 2 : c0 + 1;
+      float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+      for (int g2 = 0; g2 < kColGroups; ++g2) { sum0 += psum[g2 * 2 * D + c0]; sum1 += psum[g2 * 2 * D + c1]; }
+      if (is_k) {
+        const float cs = rope_cs[2 * u], sn = rope_cs[2 * u + 1];
+        const float x1 = sum0, x2 = sum1;
+        sum0 = fmaf(x1, cs, -x2 * sn);
+        sum1 = fmaf(x2, cs, x1 * sn);
+      }
+      kg[c0] = __bfloat162float(__float2bfloat16_rn(sum0));   // kg | vg are contiguous; values as stored
+      kg[c1] = __bfloat162float(__float2bfloat16_rn(sum1));
+    }
+    __syncthreads();
+    MASW_CLOCK(tr, 27);   // ... the new slot's key and value are final
+    if (warp < p.G) {   // scores of the G slot rows: one warp per row
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < kQPerLane; ++e)
+        dot = fmaf(__uint_as_float(static_cast<unsigned>(qraw[e]) << 16), kg[lane + 32 * e], dot);
+      for (int o2 = 16; o2 > 0; o2 >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o2);
+      if (lane == 0) sg[warp] = dot * p.scale_log2e;
+    }
+    if (split == 0) {
+      const int m_slot = p.n_slots[b];
+      if (m_slot < p.max_slots) {
+        for (int c = tid; c < 2 * D; c += NT) {
+          __nv_bfloat16* dst = (c < D ? p.k_base : p.v_base) + b * p.stride_b + kvh * p.stride_h +
+                               static_cast<long long>(p.S + m_slot) * D + (c % D);
+          *dst = __float2bfloat16_rn(kg[c]);
+        }
+      } else if (tid == 0 && p.status) {
+        atomicOr(p.status, MASW_STATUS_SLOT_OVERFLOW);
+      }
+    }
+    __syncthreads();
+    MASW_CLOCK(tr, 28);   // ... the slot phase is over
+  };
+
+  for (int base = 0; base < my_items; base += kSlots) {
+    const int li = base + tid / kGroups;      // local item
+    const int grp = tid % kGroups;
+    const bool live = li < my_items;
+    const int idx = i_begin + (live ? li : 0);
+    const int r = idx / (D / 4);
+    const int d4 = (idx % (D / 4)) * 4;
+    float m_run2 = kNegInf, l_run2 = 0.f;
+    float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    // everything the final combine needs besides the partials is worked out before the records are awaited
+    const int j = r / p.G, g = r % p.G;
+    const size_t row_off = (static_cast<size_t>(b) * p.n_q + j) * p.Hq + kvh * p.G + g;
+    float* const out_o = p.o + row_off * D + d4;
+    __nv_bfloat16* const out_bf16 = p.o_bf16 ? p.o_bf16 + row_off * D + d4 : nullptr;
+    float* const out_lse = (d4 == 0 && p.lse) ? p.lse + row_off : nullptr;
+    const bool with_slot = slot_term && idx >= first_slot_item;
+    const float* const my_gsm = gsm + (tid / kGroups) * 6;
+    if (live) {
+      for (int sp0 = grp; sp0 < splits; sp0 += kGroups * kFetch) {
+        float2 ml[kFetch];
+        float4 v[kFetch];
+        bool okv[kFetch];
+        bool all_ok = true;
+#pragma unroll
+        for (int u = 0; u < kFetch; ++u) {
+          okv[u] = true;
+          const int sp = sp0 + u * kGroups;
+          if (sp < splits) {
+            rec_fetch_item(all_ml + (sp * KROWS + r) * 2, all_o + (static_cast<size_t>(sp) * KROWS + r) * D + d4, tag, ml[u],
+                           v[u], okv[u]);
+            all_ok &= okv[u];
+          }
+        }
+        for (int it = 0; !all_ok && it < MASW_WAIT_LIMIT(p); ++it) {   // a split that has not published yet
+          __nanosleep(20);
+          all_ok = true;
+#pragma unroll
+          for (int u = 0; u < kFetch; ++u) {
+            if (!okv[u]) {
+              const int sp = sp0 + u * kGroups;
+              rec_fetch_item(all_ml + (sp * KROWS + r) * 2, all_o + (static_cast<size_t>(sp) * KROWS + r) * D + d4, tag,
+                             ml[u], v[u], okv[u]);
+              all_ok &= okv[u];
+            }
+          }
+        }
+        timed_out |= !all_ok;
+        MASW_CLOCK(tr, 11);   // developer build: thread 0 holds every split's record of its first item
+        float mb = m_run2;
+#pragma unroll
+        for (int u = 0; u < kFetch; ++u) if (sp0 + u * kGroups < splits) mb = fmaxf(mb, ml[u].x);
+        const float mu = (mb == kNegInf) ? 0.f : mb;
+        const float c = fast_exp2(m_run2 - mu);
+        o4.x *= c; o4.y *= c; o4.z *= c; o4.w *= c;
+        l_run2 *= c;
+        m_run2 = mb;
+#pragma unroll
+        for (int u = 0; u < kFetch; ++u) {
+          if (sp0 + u * kGroups < splits) {
+            const float w = fast_exp2(ml[u].x - mu);   // exp2(-inf) = 0 for an empty split
+            o4.x += w * v[u].x; o4.y += w * v[u].y; o4.z += w * v[u].z; o4.w += w * v[u].w;
+            l_run2 += w * ml[u].y;
+          }
+        }
+      }
+      float* dst = gsm + (grp * kSlots + tid / kGroups) * 6;
+      dst[0] = m_run2; dst[1] = l_run2; dst[2] = o4.x; dst[3] = o4.y; dst[4] = o4.z; dst[5] = o4.w;
+    }
+    __syncthreads();
+    MASW_CLOCK(tr, 12);     // developer build: every item of this CTA has all its records
+    if (base == 0 && slot_term) slot_phase();
+    const float s_new = with_slot ? sg[g] : 0.f;
+    const float4 v_new = with_slot ? make_float4(vg[d4], vg[d4 + 1], vg[d4 + 2], vg[d4 + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (live && grp == 0) {
+      // the groups' partials (m, l | o.x, o.y | o.z, o.w), merged in group order
+      float m = kNegInf;
+#pragma unroll
+      for (int g2 = 0; g2 < kGroups; ++g2) m = fmaxf(m, my_gsm[g2 * kSlots * 6]);
+      if (with_slot) m = fmaxf(m, s_new);
+      float l = 0.f;
+      float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int g2 = 0; g2 < kGroups; ++g2) {
+        const float2 ml2 = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6);
+        const float2 oa = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6 + 2);
+        const float2 ob = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6 + 4);
+        const float w = (ml2.x == kNegInf) ? 0.f : fast_exp2(ml2.x - m);
+        l += w * ml2.y;
+        o.x += w * oa.x; o.y += w * oa.y; o.z += w * ob.x; o.w += w * ob.y;
+      }
+      if (with_slot) {
+        const float w_new = fast_exp2(s_new - m);
+        l += w_new;
+        o.x += w_new * v_new.x; o.y += w_new * v_new.y; o.z += w_new * v_new.z; o.w += w_new * v_new.w;
+      }
+      MASW_CLOCK(tr, 21);     // developer build: combined, before the stores
+      const float inv = (l > 0.f) ? __frcp_rn(l) : 0.f;
+      o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
+      *reinterpret_cast<float4*>(out_o) = o;
+      if (out_bf16) *reinterpret_cast<uint2*>(out_bf16) = make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
+      if (out_lse) *out_lse = (l > 0.f) ? (m + __log2f(l)) * 0.6931471805599453f : kNegInf;
+    }
+    MASW_CLOCK(tr, 22);     // developer build: this CTA's outputs are stored
+    if (base + kSlots < my_items) __syncthreads();   // the group partials are overwritten by the next batch of items
+  }
+  if (timed_out && p.status) atomicOr(p.status, MASW_STATUS_WAIT_TIMEOUT);
+  // every split has published records tagged with this launch's epoch, so all of them have read the old one
+  if (split == 0 && tid == 0) p.tickets[bh * (kMaxSplitsDev + 1)] = tag;
 }
 
 template <int D>
@@ -104,6 +353,9 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #endif
   MASW_STAMP(tr, 0);
 
+#ifdef MASW_TRACE
+  if (p.debug_flags & 8) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // timing experiment: successor released at once
+#endif
   if (is_producer) {
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
@@ -188,17 +440,17 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
   };
 
-  // rotation angles of the slot this launch creates (boundary step): prepared in double by the last warp (ahead
-  // of the wait when the launch may start early), kept in registers until the stages are free to hold them
+  // rotation angles of the slot this launch creates (boundary step): formed in double by the last warp (ahead of
+  // the wait when the launch may start early); their cosine and sine are kept as fp32 in the control block
+  // (the rotated key is rounded to bf16, so fp32 factors lose nothing)
   constexpr int kRopePerLane = D / 64;
-  double rope_c[kRopePerLane], rope_s[kRopePerLane];
 
   // ---- Q^T fragments (B operand: 16 dims x 8 rows per step) straight from global memory into registers.
   // Thread (lane / 4, lane % 4) holds row lane / 4, dims 16 ks + 2 (lane % 4) + {0, 1} and + 8.
   const int gq = lane >> 2;
   const int q2 = (lane & 3) * 2;
   uint32_t qb[D / 16][2];
-  int epoch_reg = 0;   // thread 0: this head's reduction epoch, kept in a register until the publication needs it
+  int epoch_reg = 0;   // this head's reduction epoch (every thread loads it: one broadcast transaction per warp)
   auto wait_for_predecessor_and_load_q = [&]() {
     // a launch that was allowed to start early waits here for its predecessor, and lets its own successor start
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -216,18 +468,50 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         qb[ks][1] = real ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
       }
     }
-    if (tid == 0) epoch_reg = __ldcg(p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1));
+    epoch_reg = __ldcg(p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1));
+  };
+
+  // ---- fused slot materialisation, part 1 (boundary step): this CTA's slice of K_g = h_g W_K,g and V_g = h_g W_V,g
+  //      for its KV head (rows [pk0, pk1) of the d_model contraction), in registers only: warp w owns 2 D / 8 of
+  //      the head's 2 D output columns (K | V), a lane one 16-byte chunk of every (32 / chunks)-th weight row.
+  //      The mirrored projections are parameters, which no launch of a decoding step writes: with p.early their
+  //      rows are requested ahead of the wait and only h_g is read behind it.
+  constexpr int kProjColsPerWarp = 2 * D / NW;        // 16 or 32
+  constexpr int kProjChunks = kProjColsPerWarp / 8;   // 16-byte chunks of a row this warp reads: 2 or 4
+  constexpr int kProjRowLanes = 32 / kProjChunks;
+  constexpr int kProjInFlight = 8;                    // weight rows per lane and round trip
+  const bool proj_on = p.h_g != nullptr && (p.active == nullptr || p.active[b] != 0);
+  const int prl = lane / kProjChunks;
+  const int pcol = warp * kProjColsPerWarp + (lane % kProjChunks) * 8;   // first of this lane's eight columns in K | V
+  const int pk0 = static_cast<int>((static_cast<long long>(p.d_model) * split) / p.splits);
+  const int pk1 = static_cast<int>((static_cast<long long>(p.d_model) * (split + 1)) / p.splits);
+  uint4 pw[kProjInFlight];
+  auto proj_load_weights = [&](int kb) {
+    const __nv_bfloat16* W = (pcol < D ? p.Wk_g : p.Wv_g) + kvh * D + (pcol < D ? pcol : pcol - D);
+    const int ncols = p.Hkv * D;
+#pragma unroll
+    for (int u = 0; u < kProjInFlight; ++u) {
+      const int k = kb + u * kProjRowLanes;
+      pw[u] = make_uint4(0, 0, 0, 0);
+      if (k < pk1) pw[u] = __ldg(reinterpret_cast<const uint4*>(W + static_cast<size_t>(k) * ncols));
+    }
   };
 
   // Without p.early everything follows the wait.  With it, the plan and the first ring of copies come first and
   // only q, the pending raw rows and the epoch are read behind the wait: the tiles are in shared memory by then.
-  if (!p.early) wait_for_predecessor_and_load_q();
+  if (!p.early) {
+    wait_for_predecessor_and_load_q();
+    if (proj_on) proj_load_weights(pk0 + prl);
+  }
   plan_and_issue();
   if (warp == NW - 1 && p.h_g != nullptr) {
 #pragma unroll
     for (int u = 0; u < kRopePerLane; ++u) {
       const int i = lane + 32 * u;
-      sincos(static_cast<double>(p.slot_pos[b]) * pow(p.rope_base, -2.0 * i / D), &rope_s[u], &rope_c[u]);
+      double sn, cs;
+      sincos(static_cast<double>(p.slot_pos[b]) * pow(p.rope_base, -2.0 * i / D), &sn, &cs);
+      ctl->rope[2 * i] = static_cast<float>(cs);
+      ctl->rope[2 * i + 1] = static_cast<float>(sn);
     }
   }
   __syncthreads();   // the plan and the barriers are visible to every warp
@@ -324,15 +608,10 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         prefetch_l2(src);
       }
     }
-    if (p.h_g != nullptr) {
-      const int k0 = static_cast<int>((static_cast<long long>(p.d_model) * split) / p.splits);
-      const int k1 = static_cast<int>((static_cast<long long>(p.d_model) * (split + 1)) / p.splits);
-      for (int k = k0 + tid; k < k1; k += C::kThreads) {
-        const size_t off = static_cast<size_t>(k) * (p.Hkv * D) + kvh * D;
-#pragma unroll
-        for (int c = 0; c < D / 64; ++c) { prefetch_l2(p.Wk_g + off + c * 64); prefetch_l2(p.Wv_g + off + c * 64); }
-      }
-      if (tid == 0) prefetch_l2(p.h_g + static_cast<size_t>(b) * p.d_model + k0);
+    if (proj_on) {
+      // the slot token's hidden state arrives with q; the weight rows are requested here, ahead of the wait
+      for (int k = pk0 + tid * 64; k < pk1; k += C::kThreads * 64) prefetch_l2(p.h_g + static_cast<size_t>(b) * p.d_model + k);
+      proj_load_weights(pk0 + prl);
     }
     wait_for_predecessor_and_load_q();
   }
@@ -343,6 +622,48 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   float l_run[2] = {0.f, 0.f};
 #pragma unroll
   for (int i = 0; i < D / 16; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
+
+  // ---- fused slot materialisation, part 1, the arithmetic (the weight rows were requested above): h_g arrives
+  //      with q, the row lanes are summed with shuffles, and the warp publishes its columns of the split's
+  //      partial sums at once.  By the time the attention partials meet, these records have long arrived; they
+  //      are combined, rotated and used in draft_reduce_and_store.
+  if (proj_on) {
+    const __nv_bfloat16* h = p.h_g + static_cast<size_t>(b) * p.d_model;
+    float a8[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) a8[c] = 0.f;
+    for (int kb = pk0 + prl; kb < pk1; kb += kProjRowLanes * kProjInFlight) {
+      float x[kProjInFlight];
+#pragma unroll
+      for (int u = 0; u < kProjInFlight; ++u) {
+        const int k = kb + u * kProjRowLanes;
+        x[u] = (k < pk1) ? __bfloat162float(h[k]) : 0.f;
+      }
+      if (kb != pk0 + prl) proj_load_weights(kb);   // a long slice: the later batches are requested here
+      MASW_CLOCK(tr, 23);   // developer build: the projection's inputs are requested
+#pragma unroll
+      for (int u = 0; u < kProjInFlight; ++u) {
+        const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&pw[u]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const float2 f = __bfloat1622float2(w2[c]);
+          a8[2 * c] = fmaf(x[u], f.x, a8[2 * c]);
+          a8[2 * c + 1] = fmaf(x[u], f.y, a8[2 * c + 1]);
+        }
+      }
+    }
+#pragma unroll
+    for (int off = kProjChunks; off < 32; off <<= 1) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) a8[c] += __shfl_xor_sync(0xffffffffu, a8[c], off);
+    }
+    MASW_CLOCK(tr, 24);     // ... its sums are complete
+    if (prl == 0) {
+      unsigned long long* pslot = p.part_slot + (static_cast<size_t>(b * p.Hkv + kvh) * p.splits + split) * 2 * D + pcol;
+#pragma unroll
+      for (int c = 0; c < 8; c += 2) rec_store2(pslot + c, a8[c], a8[c + 1], epoch_reg + 1);
+    }
+  }
 
   // ---- Geometry of a warp's next tile, prepared one tile ahead.  Fused append: the pending raw tokens
   // (positions t .. t + n_raw - 1) are not in memory yet; the warp that owns their tile overwrites their rows of
@@ -662,7 +983,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   constexpr int kMS = C::kMergeStride;
   float* mo = reinterpret_cast<float*>(pipe + C::kMergeOff);   // [NW][8][kMS]
   float* mml = mo + NW * C::kRows * kMS;                       // [NW][8][2]
-  double* rope_cs = reinterpret_cast<double*>(pipe + C::kRopeOff);
+  const float* rope_cs = ctl->rope;
   {
     float* o0 = mo + (warp * C::kRows + q2) * kMS;
     float* o1 = o0 + kMS;
@@ -674,13 +995,6 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (gq == 0) {
       mml[(warp * C::kRows + q2) * 2 + 0] = m_run[0]; mml[(warp * C::kRows + q2) * 2 + 1] = l_run[0];
       mml[(warp * C::kRows + q2 + 1) * 2 + 0] = m_run[1]; mml[(warp * C::kRows + q2 + 1) * 2 + 1] = l_run[1];
-    }
-  }
-  if (warp == NW - 1 && p.h_g != nullptr) {
-#pragma unroll
-    for (int u = 0; u < kRopePerLane; ++u) {
-      const int i = lane + 32 * u;
-      rope_cs[2 * i] = rope_c[u]; rope_cs[2 * i + 1] = rope_s[u];
     }
   }
   __syncthreads();
@@ -715,89 +1029,16 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   }
   MASW_CLOCK(tr, 9);      // the partial is published
 
-  // ---- fused slot materialisation, part 1 (boundary step): this CTA's slice of K_g = h_g W_K,g and
-  //      V_g = h_g W_V,g for its KV head (rows [k0, k1) of the d_model contraction); the splits' partial sums
-  //      are combined, rotated and used in split_reduce_and_store.  A thread owns eight columns (one 16-byte
-  //      load per weight row) of every kRowLanes-th row.  It follows the attention partial so that the other
-  //      splits can already fetch that while the weights stream.
-  if (p.h_g != nullptr) {
-    constexpr int kColThreads = D / 8;
-    constexpr int kRowLanes = C::kThreads / kColThreads;
-    constexpr int kChunk = 4;   // weight rows per thread and round trip
-    const bool act = (p.active == nullptr) || (p.active[b] != 0);
-    const int k0 = static_cast<int>((static_cast<long long>(p.d_model) * split) / p.splits);
-    const int k1 = static_cast<int>((static_cast<long long>(p.d_model) * (split + 1)) / p.splits);
-    __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(pipe + C::kProjHsOff);     // [k1 - k0]
-    float* red = reinterpret_cast<float*>(pipe + C::kProjRedOff);                    // [kRowLanes][2 * D]
-    const int nk = min(k1 - k0, 8192);   // the staging area holds 16 KB of hidden state
-    if (act) {
-      for (int k = tid; k < nk; k += C::kThreads) hs[k] = p.h_g[static_cast<size_t>(b) * p.d_model + k0 + k];
-    }
-    __syncthreads();
-    const int ct = tid % kColThreads, rl = tid / kColThreads;
-    const int ncols = p.Hkv * D;
-    float ak[8], av[8];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) { ak[c] = 0.f; av[c] = 0.f; }
-    if (act && rl < kRowLanes) {
-      for (int kb = k0 + rl; kb < k1; kb += kRowLanes * kChunk) {
-        uint4 wk[kChunk], wv[kChunk];
-#pragma unroll
-        for (int u = 0; u < kChunk; ++u) {
-          const int k = kb + u * kRowLanes;
-          if (k < k1) {
-            const size_t off = static_cast<size_t>(k) * ncols + kvh * D + ct * 8;
-            wk[u] = __ldg(reinterpret_cast<const uint4*>(p.Wk_g + off));
-            wv[u] = __ldg(reinterpret_cast<const uint4*>(p.Wv_g + off));
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < kChunk; ++u) {
-          const int k = kb + u * kRowLanes;
-          if (k < k1) {
-            const float x = (k - k0 < nk) ? __bfloat162float(hs[k - k0])
-                                          : __bfloat162float(p.h_g[static_cast<size_t>(b) * p.d_model + k]);
-            const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&wk[u]);
-            const __nv_bfloat162* v2 = reinterpret_cast<const __nv_bfloat162*>(&wv[u]);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const float2 fk = __bfloat1622float2(k2[c]), fv = __bfloat1622float2(v2[c]);
-              ak[2 * c] = fmaf(x, fk.x, ak[2 * c]); ak[2 * c + 1] = fmaf(x, fk.y, ak[2 * c + 1]);
-              av[2 * c] = fmaf(x, fv.x, av[2 * c]); av[2 * c + 1] = fmaf(x, fv.y, av[2 * c + 1]);
-            }
-          }
-        }
-      }
-    }
-    if (rl < kRowLanes) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        red[rl * 2 * D + ct * 8 + c] = ak[c];
-        red[rl * 2 * D + D + ct * 8 + c] = av[c];
-      }
-    }
-    __syncthreads();
-    unsigned long long* pslot = p.part_slot + (static_cast<size_t>(bh) * p.splits + split) * 2 * D;
-    for (int c = tid; c < 2 * D; c += C::kThreads) {
-      float a = 0.f;
-      for (int l2 = 0; l2 < kRowLanes; ++l2) a += red[l2 * 2 * D + c];
-      rec_store1(pslot + c, a, tag);
-    }
-  }
-
 #ifdef MASW_TRACE
   if (tr && tid == 0) { tr[5] = 1; tr[6] = n_tiles; unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); tr[7] = sm; }
 #endif
-  // ---- cross-split reduction (see split_reduce_and_store)
+  // ---- cross-split reduction
 #ifdef MASW_TRACE
   if (p.debug_flags & 1) return;
+#else
+  long long* tr = nullptr;
 #endif
-  split_reduce_and_store<D, C::kRows, C::kThreads>(p, b, kvh, split, n_rows, plan[6], reinterpret_cast<float*>(pipe + C::kReduceOff),
-                                                   tid, p.h_g != nullptr ? rope_cs : nullptr
-#ifdef MASW_TRACE
-                                                   , tr
-#endif
-                                                   );
+  draft_reduce_and_store<D>(p, b, kvh, split, n_rows, plan[6], reinterpret_cast<float*>(pipe + C::kReduceOff), tid, rope_cs, tr);
   MASW_CLOCK(tr, 13);
   MASW_STAMP(tr, 4);
 }
