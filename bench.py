@@ -25,9 +25,11 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 METRIC = "draft+verify attention us/step at 32K prefix"
-# dram__bytes_read + dram__bytes_write of one verify launch divided by its KV bytes, from the ncu capture
-# summarised in profiles/attend_kernels_cfg2_full.md (34.22 MB measured for 33.575 MB of KV)
+# dram__bytes_read + dram__bytes_write of one launch divided by its KV bytes, from the ncu capture of an 8K-prefix
+# case summarised in profiles/attend_kernels_cfg2_full.md (verify: 34.03 MB for 33.575 MB of KV; draft: 4.43 MB for
+# 4.19 MB of KV, the rest being q, the pending rows and the split partials)
 NCU_TRAFFIC_RATIO = 34.03 / 33.575
+NCU_TRAFFIC_RATIO_DRAFT = 4.43 / 4.194
 UNIT = "us/step"
 TRACE_WORDS = 32   # 64-bit words per CTA in the developer build's stamp records
 SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -545,20 +547,39 @@ def run_gpu(args, wl):
     if clocks is not None:   # more warm-up steps until the clock sampler is up
         clocks.wait_first(lambda: (runner.step_resident(), torch.cuda.synchronize()))
     barrier()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # The block of exactly K steps is repeated until about half a second has been timed (so that the clock
+    # sampler has samples inside the region); the reported step time is the median block, with the spread beside it.
+    probe0, probe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    probe0.record(); runner.step_resident(); probe1.record(); barrier()
+    n_blocks = int(min(40, max(1, round(args.min_timed_s * 1e3 / max(probe0.elapsed_time(probe1) * K, 1e-3)))))
+    if world > 1:   # every rank must run the same number of blocks
+        nb = torch.tensor([n_blocks], dtype=torch.int64, device=dev)
+        dist.all_reduce(nb, op=dist.ReduceOp.MAX)
+        n_blocks = int(nb.item())
+    block_ms, phase_blocks = [], []
     if clocks is not None:
         clocks.begin()
-    start.record()
-    for i in range(K):
-        runner.step_resident(evs[i])
-    stop.record()
-    barrier()
+    for _ in range(n_blocks):
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for i in range(K):
+            runner.step_resident(evs[i])
+        stop.record()
+        barrier()
+        block_ms.append(start.elapsed_time(stop))
+        phase_blocks.append([sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(3)])
     if clocks is not None:
         clocks.end()
     clock_info = clocks.stop() if rank == 0 else None
-    total_ms = start.elapsed_time(stop)
-    phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(3)]
+    order = sorted(range(n_blocks), key=lambda i: block_ms[i])
+    mid = order[(n_blocks - 1) // 2]
+    total_ms = block_ms[mid]
+    phase_ms = phase_blocks[mid]
+    block_stats = {"blocks": n_blocks, "steps_per_block": K, "us_per_step_median": block_ms[mid] * 1e3 / K,
+                   "us_per_step_min": min(block_ms) * 1e3 / K, "us_per_step_max": max(block_ms) * 1e3 / K,
+                   "timed_s": sum(block_ms) / 1e3}
 
     # ---- end-to-end timing through host buffers
     for _ in range(W):
@@ -588,6 +609,10 @@ def run_gpu(args, wl):
         peak, peak_kind = measured_peak_gbs()
         v_gbs = verify_bytes / (verify_us * 1e-6) / 1e9
         d_gbs = draft_bytes_step / (draft_us * 1e-6) / 1e9
+        draft_bytes_layer = wl.draft_kv_bytes_per_layer()
+        draft_launch_us = draft_us / wl.d_layers               # mean over plain, boundary and first-of-step launches
+        step_bytes = draft_bytes_step * g + verify_bytes
+        step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
         base = cpu_baseline(wl) if world == 1 and not args.no_cpu_baseline else None
         comp = None
         kinds = draft_launch_kinds(runner) if world == 1 else None
@@ -623,10 +648,23 @@ def run_gpu(args, wl):
                          "traffic_source": "ncu dram bytes of an 8K-prefix launch (profiles/attend_kernels_cfg2_full.md) "
                                            "scaled by KV bytes; traffic grows in proportion to the entries",
                          "algorithmic_bytes_per_launch": verify_bytes_layer,
-                         "launches_timed": wl.t_layers * K, "avg_launch_us": verify_us / wl.t_layers},
+                         "launches_timed": wl.t_layers * K * n_blocks, "avg_launch_us": verify_us / wl.t_layers},
+            # the other half of the step: the draft's decode launch (16.8 MB of KV per launch at batch 1, latency-bound)
+            "roofline_draft": {"kernel": "attend_draft_kernel (draft_append_attend / draft_boundary_attend, one draft layer per launch)",
+                               "bound": "hbm", "achieved": d_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                               "frac": d_gbs / peak, "frac_of_8tbs": d_gbs / 8000.0,
+                               "traffic": draft_bytes_layer * NCU_TRAFFIC_RATIO_DRAFT,
+                               "traffic_source": "ncu dram bytes of an 8K-prefix launch (profiles/attend_kernels_cfg2_full.md) "
+                                                 "scaled by KV bytes",
+                               "algorithmic_bytes_per_launch": draft_bytes_layer,
+                               "launches_timed": wl.d_layers * g * K * n_blocks, "avg_launch_us": draft_launch_us},
+            # the whole iteration against the same peak: all KV bytes of the step over the step time
+            "step_frac": {"kv_bytes_per_step": step_bytes, "achieved": step_gbs, "peak": peak, "unit": "GB/s",
+                          "frac": step_gbs / peak, "frac_of_8tbs": step_gbs / 8000.0},
+            "timing": block_stats,
             "e2e": {"value": job_value_us(e2e_ms / K, world), "unit": UNIT, "h2d_bytes_per_step": in_bytes,
                     "d2h_bytes_per_step": out_bytes, "wall_us_per_step": e2e_wall_ms * 1e3 / K},
-            "gpu_launches": launches_per_step * K,
+            "gpu_launches": launches_per_step * K * n_blocks,     # kernels launched inside the timed blocks
             "gpu_launches_per_step": launches_per_step,
             "clocks": clock_info,
             "device_status": status,
@@ -925,6 +963,8 @@ def main():
     ap.add_argument("--workload", default="cfg3_8b_32k", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--impl", default="masw", choices=["masw", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-timed-s", type=float, default=0.5,
+                    help="the block of --steps steps is repeated until about this many seconds are timed (median block reported)")
     ap.add_argument("--sweep", action="store_true", help="run the prefix x batch x gamma x ratio sweep (one JSON line per point)")
     ap.add_argument("--prefill", action="store_true",
                     help="time the draft's masked prefill pass (one layer per step) instead of the decoding iteration")
