@@ -828,6 +828,59 @@ def run_prefill(args, wl):
     print(json.dumps(row), flush=True)
 
 
+def run_loop(args):
+    """The packaged speculative-decoding loop (paper_2608_30252_b200.loop) on its toy one-layer models: greedy
+    decoding of 256 tokens after a 2000-token prompt, gamma = 5, draft memory S = 4, W = 256, r = 8.  Prints one JSON
+    line: emitted tokens per iteration, the measured draft-step and verification times, the target's one-token
+    time, Eq. 1 evaluated on those measurements, and whether the output equals target-only greedy decoding."""
+    import torch
+    from paper_2608_30252_b200 import build, binding, loop
+    if not torch.cuda.is_available():
+        raise RuntimeError("the loop benchmark needs a CUDA device")
+    torch.cuda.set_device(0)
+    build.build()
+    binding.load()
+    gamma, n, P = 5, 256, 2000
+    g0 = torch.Generator(device="cuda").manual_seed(5)
+    prompt = [int(x) for x in torch.randint(0, 64, (P,), generator=g0, device="cuda").tolist()]
+    mk_t = lambda: loop.ToyTarget(torch.Generator(device="cuda").manual_seed(1), cap=P + n + 64)
+    mk_d = lambda seed: loop.ToyDraft(torch.Generator(device="cuda").manual_seed(seed), S=4, W=256, r=8, max_pos=P + n + 64)
+    l0 = binding.launch_count()
+    ar_timer = loop.EventTimer()
+    ref = loop.greedy_target_only(mk_t(), prompt, n, timer=ar_timer)
+    t_ar = ar_timer.mean_us()
+    rows = {}
+    for name, draft, spoil in (("independent_random_draft", mk_d(7), None),
+                               ("draft_right_four_times_in_five", mk_d(7), True)):
+        res = loop.speculative(mk_t(), draft, prompt, n, gamma) if spoil is None else \
+            _run_spoiled(loop, mk_t(), draft, prompt, n, gamma, ref)
+        rows[name] = {"tok_per_iter": res.tok_per_iter, "t_d_us": res.t_d_us, "t_t_us": res.t_t_us,
+                      "eq1_speedup": res.eq1_speedup, "iterations": len(res.accepted),
+                      "equals_target_only_greedy": res.tokens == ref, "status": res.status}
+    print(json.dumps({"metric": "speculative-decoding loop on toy models", "unit": "tokens per iteration / us", "n_gpus": 1,
+                      "config": {"workload": "toy 1-layer target (8q/2kv d128) + toy 1-layer MASW draft (8q/2kv d64, S=4 W=256 r=8)",
+                                 "prompt": P, "new_tokens": n, "gamma": gamma},
+                      "target_one_token_us": t_ar, "drafts": rows, "gpu_launches": binding.launch_count() - l0,
+                      "note": "t_d and t_t include the toy models' dense layers (torch matmuls) and host-side launch gaps: "
+                              "the loop is driven eagerly from Python, so these times are launch-bound and say nothing "
+                              "about the kernels' bandwidth"}), flush=True)
+
+
+def _run_spoiled(loop, target, draft, prompt, n, gamma, ref):
+    """The draft's proposals replaced by the true continuation except every fifth one (a draft that is right four
+    times in five), so that Tok./Iter and Eq. 1 are exercised at a realistic acceptance rate."""
+    state = {"count": 0}
+
+    def spoil(it, j, tok):
+        # position of this proposal in the emitted sequence: reconstructed from the target's cache length
+        pos = target.n - len(prompt) + 1 + j
+        truth = ref[pos] if pos < len(ref) else 0
+        state["count"] += 1
+        return (truth + 1) % 64 if state["count"] % 5 == 0 else truth
+
+    return loop.speculative(target, draft, prompt, n, gamma, spoil=spoil)
+
+
 def run_timeline(args, wl):
     """Per-CTA phase timelines of one draft launch, one boundary launch and one verify launch of `wl`, from
     the %globaltimer stamps of the library's developer hook (eager launches, microseconds from the first
@@ -968,6 +1021,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the prefix x batch x gamma x ratio sweep (one JSON line per point)")
     ap.add_argument("--prefill", action="store_true",
                     help="time the draft's masked prefill pass (one layer per step) instead of the decoding iteration")
+    ap.add_argument("--loop", action="store_true",
+                    help="run the packaged speculative-decoding loop on its toy models: Tok./Iter, t_d, t_t, Eq. 1")
     ap.add_argument("--timeline", action="store_true",
                     help="per-CTA phase timelines of one draft, one boundary and one verify launch (developer stamps)")
     ap.add_argument("--traffic-bytes", type=float, default=None,
@@ -976,6 +1031,8 @@ def main():
     wl = inputs.WORKLOADS[args.workload]
     if args.sweep:
         run_sweep(args)
+    elif args.loop:
+        run_loop(args)
     elif args.timeline:
         run_timeline(args, wl)
     elif args.prefill:

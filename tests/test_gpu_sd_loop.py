@@ -1,7 +1,9 @@
-"""End-to-end speculative decoding through the C ABI on a toy one-layer target and a toy memory-augmented
-draft: greedy speculative decoding must emit exactly the target-only greedy sequence (Section 3.1 /
-Section 4.3: verification keeps the output unchanged), whatever the draft proposes, including across
-rejections, rollbacks (Section 4.3, "Rollback"), slot materialisation at boundaries and window eviction.
+"""End-to-end speculative decoding through the C ABI with the packaged loop driver (paper_2608_30252_b200.loop) on
+a toy one-layer target and a toy memory-augmented draft: greedy speculative decoding must emit exactly the
+target-only greedy sequence (Section 3.1 / Section 4.3: verification keeps the output unchanged), whatever the
+draft proposes, including across rejections, rollbacks (Section 4.3, "Rollback"), slot materialisation at
+boundaries and window eviction; and the emitted sequence is checked against a host-side copy of the same toy
+target built from the oracle's verification attention.
 
 The dense layers around the attention calls (embeddings, q/k/v projections, unembedding) are plain torch
 matmuls: the backbone is outside the library.  Everything the library owns — draft memory update, draft
@@ -10,148 +12,34 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_30252_b200 import binding
+from paper_2608_30252_b200.loop import ToyDraft, ToyTarget, greedy_target_only, sd_speedup, speculative
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-class ToyTarget:
-    def __init__(self, gen, V=64, Hq=8, Hkv=2, D=128, cap=512):
-        d = 256
-        self.V, self.Hq, self.Hkv, self.D, self.cap, self.d = V, Hq, Hkv, D, cap, d
-        r = lambda *s: torch.randn(*s, generator=gen, device=DEV)
-        self.E, self.Pos = r(V, d), r(cap, d) * 0.5
-        self.Wq, self.Wk, self.Wv = r(d, Hq * D) / d ** 0.5, r(d, Hkv * D) / d ** 0.5, r(d, Hkv * D) / d ** 0.5
-        self.Wu = r(Hq * D, V) * 2.0
-        self.K = torch.zeros((1, Hkv, cap, D), dtype=torch.bfloat16, device=DEV)
-        self.Vc = torch.zeros_like(self.K)
-        self.n = 0                                      # tokens whose K/V are in the cache
-        self.ws = {}
-
-    def logits_rows(self, tokens):
-        """Append `tokens` to the cache and return their next-token logits rows (bf16-rounded)."""
-        T = len(tokens)
-        pos = torch.arange(self.n, self.n + T, device=DEV)
-        x = self.E[torch.tensor(tokens, device=DEV)] + self.Pos[pos]
-        k = (x @ self.Wk).view(T, self.Hkv, self.D).to(torch.bfloat16)
-        v = (x @ self.Wv).view(T, self.Hkv, self.D).to(torch.bfloat16)
-        self.K[0, :, self.n:self.n + T] = k.permute(1, 0, 2)
-        self.Vc[0, :, self.n:self.n + T] = v.permute(1, 0, 2)
-        q = (x @ self.Wq).view(1, T, self.Hq, self.D).to(torch.bfloat16).contiguous()
-        kv_len = torch.tensor([self.n + T], dtype=torch.int32, device=DEV)
-        if T not in self.ws:
-            self.ws[T] = binding.verify_workspace(self.K, kv_len, self.Hq, T)
-        o, _ = binding.verify_attend(self.K, self.Vc, kv_len, q, workspace=self.ws[T])
-        self.n += T
-        return (o.view(T, -1) @ self.Wu).to(torch.bfloat16)
-
-    def truncate(self, n):
-        self.n = n
-
-
-class ToyDraft:
-    """A one-layer draft with the three-part memory: sinks, slots (adaptor = mirrored K/V projections
-    applied to the running mean of the recent inputs), local window."""
-
-    def __init__(self, gen, V=64, Hq=8, Hkv=2, D=64, S=2, W=8, r=4):
-        d = Hq * D
-        self.V, self.Hq, self.Hkv, self.D, self.S, self.W, self.r, self.d = V, Hq, Hkv, D, S, W, r, d
-        rn = lambda *s: torch.randn(*s, generator=gen, device=DEV)
-        self.E, self.Pos = rn(V, d), rn(512, d) * 0.5
-        self.Wq, self.Wk, self.Wv = rn(d, Hq * D) / d ** 0.5, rn(d, Hkv * D) / d ** 0.5, rn(d, Hkv * D) / d ** 0.5
-        self.Wkg, self.Wvg = self.Wk.to(torch.bfloat16).contiguous(), self.Wv.to(torch.bfloat16).contiguous()   # copy-init
-        self.Wu = rn(Hq * D, V) * 2.0
-        cfg = binding.MaswConfig(1, 1, Hq, Hkv, D, d, S, W, r, rollback=8, max_slots=128, gamma_max=8)
-        self.mem = binding.DraftMemory(cfg, DEV)
-        self.t = 0                                      # committed tokens (host mirror)
-        self.slots = 0
-
-    def step(self, tokens):
-        """Feed the pending tokens (their positions are t .. t+n-1), return the arg-max next token after the
-        last.  The tokens go in chunks that end at slot boundaries (and hold at most 4 tokens)."""
-        nxt = None
-        while tokens:
-            n = 1
-            while n < min(len(tokens), 4) and not self._boundary(self.t + n):
-                n += 1
-            nxt = self._step_chunk(tokens[:n])
-            tokens = tokens[n:]
-        return nxt
-
-    def _boundary(self, t_after):
-        return t_after > self.S and (t_after - self.S) % self.r == 0
-
-    def _step_chunk(self, tokens):
-        n = len(tokens)
-        pos = torch.arange(self.t, self.t + n, device=DEV)
-        x = self.E[torch.tensor(tokens, device=DEV)] + self.Pos[pos]
-        k = (x @ self.Wk).view(1, n, self.Hkv, self.D).to(torch.bfloat16).contiguous()
-        v = (x @ self.Wv).view(1, n, self.Hkv, self.D).to(torch.bfloat16).contiguous()
-        t_after = self.t + n
-        boundary = self._boundary(t_after)
-        q_rows = [x @ self.Wq]
-        if boundary:
-            h_g = x.mean(0, keepdim=True).to(torch.bfloat16).contiguous()
-            self.mem.mem_update(0, h_g=h_g, Wk_g=self.Wkg, Wv_g=self.Wvg,
-                                slot_pos=torch.tensor([t_after], dtype=torch.int32, device=DEV))
-            q_rows.append(h_g.float() @ self.Wq)
-        q = torch.cat(q_rows).view(1, -1, self.Hq, self.D).to(torch.bfloat16).contiguous()
-        o, _ = self.mem.draft_append_attend(0, k, v, q, last_row_is_slot=boundary)
-        self.mem.mem_advance(n, add_slot=boundary)
-        self.t = t_after
-        self.slots += int(boundary)
-        logits = o[0, n - 1].reshape(-1) @ self.Wu
-        return int(torch.argmax(logits))
-
-    def rollback(self, t_keep):
-        slots_keep = max(0, t_keep - self.S) // self.r
-        self.mem.mem_rollback(torch.tensor([t_keep], dtype=torch.int32, device=DEV),
-                              torch.tensor([slots_keep], dtype=torch.int32, device=DEV), slots_keep_max=slots_keep)
-        self.t, self.slots = t_keep, slots_keep
-
-
-def greedy_target_only(target, prompt, n):
-    rows = target.logits_rows(prompt)
-    out = [int(torch.argmax(rows[-1].float()))]
-    while len(out) < n:
-        out.append(int(torch.argmax(target.logits_rows([out[-1]])[0].float())))
-    return out
-
-
-def speculative(target, draft, prompt, n, gamma, spoil=None):
-    rows = target.logits_rows(prompt)                       # prefill (all prompt tokens cached)
-    emitted = [int(torch.argmax(rows[-1].float()))]
-    draft.step(prompt)                                      # draft-side prefill through the same update path, chunked
-    pending = [emitted[-1]]                                 # tokens the draft has not processed yet
-    iters, accepted_hist = 0, []
-    while len(emitted) < n:
-        t0 = draft.t
-        props = []
-        feed = list(pending)
-        for j in range(gamma):
-            tok = draft.step(feed)
-            if spoil is not None:
-                tok = spoil(iters, j, tok)
-            props.append(tok)
-            feed = [tok]
-        n_cached = target.n
-        rows = target.logits_rows([emitted[-1]] + props)    # gamma + 1 rows: last emitted token + the proposals
-        n_acc, out = binding.accept_reject(rows.view(1, gamma + 1, -1).contiguous(), None,
-                                           torch.tensor([props], dtype=torch.int32, device=DEV), None, 0.0)
-        n_acc = int(n_acc.item())
-        new = [int(x) for x in out[0, : n_acc + 1].tolist()]
-        emitted += new
-        accepted_hist.append(n_acc)
-        target.truncate(n_cached + 1 + n_acc)               # keep the last emitted token and the accepted proposals
-        # draft keeps the tokens it processed that are still on the accepted path: pending + accepted[:gamma-1]
-        keep = t0 + len(pending) + min(n_acc, gamma - 1)
-        draft.rollback(keep)
-        pending = ([props[-1]] if n_acc == gamma else []) + [new[-1]]
-        iters += 1
-    _, _, status = draft.mem.mem_get_state()
-    assert status == 0
-    return emitted[:n], accepted_hist
+def _oracle_margins(target, prompt, emitted):
+    """A host-side copy of the toy target (same weights, fp64, attention = oracle.verify_attend over the bf16 cache
+    values) scores every emitted position, teacher-forced on the emitted tokens.  Returns, per emitted token, how far
+    the oracle's logit of that token lies below the oracle's best logit (0 where the oracle picks the same token)."""
+    f = lambda t: t.double().cpu().numpy()
+    E, Pos, Wq, Wk, Wv, Wu = map(f, (target.E, target.Pos, target.Wq, target.Wk, target.Wv, target.Wu))
+    toks = list(prompt) + list(emitted[:-1])
+    x = E[np.asarray(toks)] + Pos[: len(toks)]
+    rb = oracle.round_to_bf16
+    # the GPU side forms x W in fp32 and rounds to bf16: fp64 then bf16 differs from that on rare rounding ties only
+    K = rb((x @ Wk).astype(np.float32).astype(np.float64)).reshape(1, -1, target.Hkv, target.D).transpose(0, 2, 1, 3)
+    V = rb((x @ Wv).astype(np.float32).astype(np.float64)).reshape(1, -1, target.Hkv, target.D).transpose(0, 2, 1, 3)
+    margins = []
+    for i, tok in enumerate(emitted):
+        n = len(prompt) + i                                   # cache entries this row sees: tokens 0 .. n-1
+        q = rb((x[n - 1:n] @ Wq).astype(np.float32).astype(np.float64)).reshape(1, 1, target.Hq, target.D)
+        o, _ = oracle.verify_attend(q, K[:, :, :n], V[:, :, :n], [n])
+        logits = o.reshape(-1) @ Wu
+        margins.append(float(logits.max() - logits[tok]))
+    return margins
 
 
 def test_greedy_speculative_decoding_equals_target_only_decoding():
@@ -161,16 +49,26 @@ def test_greedy_speculative_decoding_equals_target_only_decoding():
     ref = greedy_target_only(ToyTarget(torch.Generator(device=DEV).manual_seed(1)), prompt, n)
     for gamma in (3, 5):
         # (a) the memory-augmented draft's own proposals (a different random model: mostly rejected)
-        out, hist = speculative(ToyTarget(torch.Generator(device=DEV).manual_seed(1)),
-                                ToyDraft(torch.Generator(device=DEV).manual_seed(7)), prompt, n, gamma)
-        assert out == ref, (gamma, "draft")
+        res = speculative(ToyTarget(torch.Generator(device=DEV).manual_seed(1)),
+                          ToyDraft(torch.Generator(device=DEV).manual_seed(7)), prompt, n, gamma)
+        assert res.tokens == ref and res.status == 0, (gamma, "draft")
+        assert res.tok_per_iter == sum(res.accepted) / len(res.accepted) + 1
+        assert res.t_d_us > 0 and res.t_t_us > 0
+        assert abs(res.eq1_speedup - oracle.sd_speedup(res.tok_per_iter - 1, gamma, res.t_d_us, res.t_t_us)) < 1e-9
         # (b) proposals overwritten with the true continuation except every third one: long accepted runs,
         #     full acceptance (bonus token) and mid-block rejections all occur
-        out2, hist2 = speculative(ToyTarget(torch.Generator(device=DEV).manual_seed(1)),
-                                  ToyDraft(torch.Generator(device=DEV).manual_seed(7)), prompt, n, gamma,
-                                  spoil=_make_spoiler(ref, gamma))
-        assert out2 == ref, (gamma, "spoiled")
+        res2 = speculative(ToyTarget(torch.Generator(device=DEV).manual_seed(1)),
+                           ToyDraft(torch.Generator(device=DEV).manual_seed(7)), prompt, n, gamma,
+                           spoil=_make_spoiler(ref, gamma))
+        hist2 = res2.accepted
+        assert res2.tokens == ref and res2.status == 0, (gamma, "spoiled")
         assert max(hist2) == gamma and min(hist2) < gamma and len(set(hist2)) >= 2
+        assert res2.tok_per_iter > res.tok_per_iter          # the better draft emits more tokens per iteration (Eq. 1's numerator)
+    # the oracle's copy of the toy target, teacher-forced on the emitted tokens: it picks the same token everywhere
+    # except where its two best logits are closer than the bf16 rounding of the logits the decision was taken on
+    margins = _oracle_margins(ToyTarget(torch.Generator(device=DEV).manual_seed(1)), prompt, ref)
+    assert max(margins) <= 0.25, max(margins)
+    assert sum(m == 0.0 for m in margins) >= 0.95 * len(margins)
 
 
 def _make_spoiler(ref, gamma):
