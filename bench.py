@@ -172,8 +172,10 @@ class StepRunner:
         wl = self.wl
         vq = self.view("vq")
         for l in range(wl.t_layers):
+            # the caches are resident and static here: no kernel in the stream writes them (stable_cache)
             self.binding.verify_attend(self.tK[l], self.tV[l], self.kv_len, vq[l], workspace=self.v_ws, out=self.v_o[l],
-                                       lse=self.v_lse[l])
+                                       lse=self.v_lse[l], stable_cache=True,
+                                       next_kv=(self.tK[l + 1], self.tV[l + 1]) if l + 1 < wl.t_layers else None)
 
     def tail_phase(self):
         self.binding.accept_reject(self.view("tl"), None, self.view("toks"), None, 0.0, workspace=self.a_ws,
@@ -987,6 +989,48 @@ def run_timeline(args, wl):
         capture_chain()
     if 2 * (wl.d_q_heads // wl.d_kv_heads) <= 8:
         capture_chain(boundary=True)
+
+    def capture_verify_chain(n_launch=5, reps=3):
+        """Consecutive target layers replayed from one CUDA graph, one record area per launch (global-timer stamps)."""
+        stride = n_cta_max * TRACE_WORDS
+        cbuf = torch.zeros(n_launch * stride, dtype=torch.int64, device=dev)
+        vq = r.view("vq")
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+
+        def launch(l):
+            r.binding.verify_attend(r.tK[l], r.tV[l], r.kv_len, vq[l], workspace=r.v_ws, out=r.v_o[l], lse=r.v_lse[l],
+                                    stable_cache=True)
+
+        with torch.cuda.stream(side):
+            for l in range(n_launch):
+                launch(l)
+            torch.cuda.synchronize()
+            binding.debug_set_trace(cbuf, stride)
+            with torch.cuda.graph(g, stream=side):
+                for l in range(n_launch):
+                    launch(l)
+            binding.debug_set_trace(None)
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(reps):
+            cbuf.zero_()
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+        t = cbuf.cpu().numpy().reshape(n_launch, n_cta_max, TRACE_WORDS)
+        t0 = t[0][t[0][:, 4] > 0][:, 0].min()
+        for k_ in range(n_launch):
+            live = t[k_][t[k_][:, 4] > 0]
+            cols = (live[:, [0, 10, 1, 8, 9, 3, 4]] - t0) / 1000.0
+            print(json.dumps({"verify_chain_launch": k_, "ctas": int(live.shape[0]), "tiles_per_cta_min_max": [int(live[:, 6].min()), int(live[:, 6].max())],
+                              "unit": "us from the first launch's first CTA: median (min-max)",
+                              **{name: f"{np.median(cols[:, c]):.2f} ({cols[:, c].min():.2f}-{cols[:, c].max():.2f})"
+                                 for c, name in enumerate(["cta_start", "wait_passed", "prologue_done", "softmax_loop_end",
+                                                           "partial_published", "before_reduce", "end"])}}), flush=True)
+
+    if wl.t_head_dim == 128:
+        capture_verify_chain()
 
     L = min(3, wl.d_layers - 1)
     q1, q2 = r.view("dq0"), r.view(f"dq{r.slot_step}")

@@ -95,6 +95,11 @@ typedef struct masw_kv_desc {
   float softmax_scale;       /* 0 selects 1 / sqrt(D) */
   int32_t flags;             /* MASW_KV_* bits, 0 for the defaults */
   int32_t* status;           /* [device] one int32 that receives MASW_STATUS_* bits (OR-ed in), or NULL */
+  const void* next_k;        /* [device] optional hint (verify_attend, head_dim 128): K and V of the cache the NEXT call */
+  const void* next_v;        /*   will read (the next layer's; same geometry and strides), or NULL.  When its own tiles
+                                  are all requested, each CTA asks for the first tile it will stream in that call to be
+                                  brought into L2, so the next launch does not start on a cold DRAM round trip.  Only a
+                                  hint: nothing is read through these pointers. */
 } masw_kv_desc;
 
 /* masw_kv_desc.flags / masw_paged_kv_desc.flags */
@@ -103,7 +108,13 @@ enum {
    * of a head claim tiles from a shared pool.  A repeated call on the same inputs then returns the same
    * bits (the pooled schedule only agrees within the rounding of the bf16 probabilities), a little slower
    * because every split waits for the slowest SM. */
-  MASW_KV_DETERMINISTIC = 1
+  MASW_KV_DETERMINISTIC = 1,
+  /* verify_attend, head_dim 128, contiguous cache: the caller vouches that the kernel which precedes this call
+   * in the stream writes nothing of the K and V arrays (the T new rows were appended by an earlier kernel, or
+   * the cache is static as in a benchmark).  The launch may then request its first K/V tiles before it waits
+   * for that kernel; q, kv_len and the scratch are still read behind the wait.  Without the flag everything is
+   * read behind the wait. */
+  MASW_KV_STABLE = 2
 };
 
 /* ---------------------------------------------------------------------------------------------------

@@ -18,6 +18,7 @@ MASW_OK, MASW_EINVAL, MASW_EALIGN, MASW_ECAPACITY, MASW_ESTATE, MASW_ECUDA = 0, 
 STATUS_SLOT_OVERFLOW, STATUS_WAIT_TIMEOUT, STATUS_BAD_LOGIT, STATUS_BAD_TOKEN = 1, 2, 4, 8
 REGION_SINK, REGION_SLOT, REGION_LOCAL = 0, 1, 2
 KV_DETERMINISTIC = 1
+KV_STABLE = 2
 
 EXPORTED_SYMBOLS = [
     "masw_sizes", "mem_init", "mem_free", "mem_load", "mem_set_state", "mem_get_state", "mem_update",
@@ -43,7 +44,7 @@ class masw_kv_desc(C.Structure):
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64),
                 ("stride_n", C.c_int64), ("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("capacity", C.c_int32), ("kv_len", C.c_void_p), ("softmax_scale", C.c_float),
-                ("flags", C.c_int32), ("status", C.c_void_p)]
+                ("flags", C.c_int32), ("status", C.c_void_p), ("next_k", C.c_void_p), ("next_v", C.c_void_p)]
 
 
 _lib = None
@@ -302,12 +303,13 @@ DraftMemory.draft_prefill_slots = _draft_prefill_slots
 DraftMemory.draft_prefill_attend = _draft_prefill_attend
 
 
-def _kv_desc(k, v, kv_len, n_q_heads, softmax_scale=0.0, flags=0, status=None) -> masw_kv_desc:
+def _kv_desc(k, v, kv_len, n_q_heads, softmax_scale=0.0, flags=0, status=None, next_kv=None) -> masw_kv_desc:
     assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.stride() == v.stride() and k.stride(-1) == 1
     assert kv_len.dtype == torch.int32 and (status is None or status.dtype == torch.int32)
     B, Hkv, cap, D = k.shape
     return masw_kv_desc(k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2), B, n_q_heads, Hkv, D, cap,
-                        kv_len.data_ptr(), softmax_scale, flags, None if status is None else status.data_ptr())
+                        kv_len.data_ptr(), softmax_scale, flags, None if status is None else status.data_ptr(),
+                        None if next_kv is None else next_kv[0].data_ptr(), None if next_kv is None else next_kv[1].data_ptr())
 
 
 def verify_workspace(k, kv_len, n_q_heads, T) -> torch.Tensor:
@@ -318,12 +320,15 @@ def verify_workspace(k, kv_len, n_q_heads, T) -> torch.Tensor:
 
 
 def verify_attend(k, v, kv_len, q, workspace=None, out=None, lse=None, out_bf16=None, softmax_scale=0.0,
-                  deterministic=False, status=None, lib=None):
+                  deterministic=False, stable_cache=False, status=None, next_kv=None, lib=None):
     """k, v: bf16 [B, Hkv, cap, D] views; kv_len int32 [B] (including the T rows); q bf16 [B, T, Hq, D].
-    deterministic: static tile schedule (bitwise repeatable); status: int32 [1] device tensor for MASW_STATUS_* bits."""
+    deterministic: static tile schedule (bitwise repeatable); stable_cache: the preceding kernel in the stream writes
+    nothing of k and v (first tiles requested ahead of the wait); status: int32 [1] device tensor for MASW_STATUS_* bits;
+    next_kv: (k, v) of the cache the next call will read (same geometry), an L2 hint for that call's first tiles."""
     assert q.dtype == torch.bfloat16 and q.is_contiguous()
     B, T, Hq, D = q.shape
-    desc = _kv_desc(k, v, kv_len, Hq, softmax_scale, KV_DETERMINISTIC if deterministic else 0, status)
+    desc = _kv_desc(k, v, kv_len, Hq, softmax_scale,
+                    (KV_DETERMINISTIC if deterministic else 0) | (KV_STABLE if stable_cache else 0), status, next_kv)
     if workspace is None:
         workspace = verify_workspace(k, kv_len, Hq, T)
     if out is None:

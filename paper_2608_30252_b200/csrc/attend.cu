@@ -109,8 +109,8 @@ static int launch_attend_draft(const CUtensorMap& tmK, const CUtensorMap& tmV, A
 
 // tcgen05 / TMEM kernel (head_dim 128): query rows padded to NQ, rings of NK K tiles and NV V tiles (32 KB each)
 template <int NQ, int NK, int NV>
-static int launch_attend_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendParams p, int B, int Hkv,
-                            int tiles_upper, int splits_max, cudaStream_t st) {
+static int launch_attend_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmKn, const CUtensorMap& tmVn,
+                            AttendParams p, int B, int Hkv, int tiles_upper, int splits_max, cudaStream_t st) {
   using C = TcCfg<NQ, NK, NV>;
   auto kern = attend_tc_kernel<NQ, NK, NV>;
   static PerDeviceOnce once;
@@ -133,7 +133,7 @@ static int launch_attend_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, Atte
   attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[na].val.programmaticStreamSerializationAllowed = 1; ++na;
   cfg.attrs = attr;
   cfg.numAttrs = na;
-  MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmK, tmV, p));
+  MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmK, tmV, tmKn, tmVn, p));
   count_launch();
   return MASW_OK;
 }
@@ -368,6 +368,7 @@ extern "C" int verify_attend(const masw_kv_desc* kv, const void* q, int T, float
   p.tickets = reinterpret_cast<int*>(ws + w.off_tickets);
   p.status = kv->status;
   p.deterministic = (kv->flags & MASW_KV_DETERMINISTIC) ? 1 : 0;
+  p.early = (kv->flags & MASW_KV_STABLE) ? 1 : 0;
   p.t = nullptr; p.n_slots = nullptr; p.kv_len = kv->kv_len;
   p.n_q = T; p.last_row_is_slot = 0;
   p.G = G; p.Hq = kv->n_q_heads; p.Hkv = kv->n_kv_heads;
@@ -377,9 +378,19 @@ extern "C" int verify_attend(const masw_kv_desc* kv, const void* q, int T, float
   p.scale_log2e = scale * 1.4426950408889634f;
   if (use_tc) {
     const int tiles_upper = (kv->capacity + 127) / 128;
+    // the next call's cache (an L2 hint): its tensor maps, or this call's own when there is none (never used then)
+    CUtensorMap tkn = tk, tvn = tv;
+    p.next_hint = 0;
+    if (kv->next_k != nullptr && kv->next_v != nullptr && aligned16(kv->next_k) && aligned16(kv->next_v)) {
+      masw_kv_desc nx = *kv;
+      nx.k = kv->next_k; nx.v = kv->next_v;
+      rc = get_kv_maps(nx, 128, &tkn, &tvn);
+      if (rc != MASW_OK) return rc;
+      p.next_hint = 1;
+    }
     if (T * G <= 32)
-      return launch_attend_tc<32, 3, 3>(tk, tv, p, kv->batch, kv->n_kv_heads, tiles_upper, w.splits_max, static_cast<cudaStream_t>(stream));
-    return launch_attend_tc<64, 2, 3>(tk, tv, p, kv->batch, kv->n_kv_heads, tiles_upper, w.splits_max, static_cast<cudaStream_t>(stream));
+      return launch_attend_tc<32, 3, 3>(tk, tv, tkn, tvn, p, kv->batch, kv->n_kv_heads, tiles_upper, w.splits_max, static_cast<cudaStream_t>(stream));
+    return launch_attend_tc<64, 2, 3>(tk, tv, tkn, tvn, p, kv->batch, kv->n_kv_heads, tiles_upper, w.splits_max, static_cast<cudaStream_t>(stream));
   }
   return dispatch_attend(kv->head_dim, mt, tk, tv, p, kv->batch, kv->n_kv_heads, kv->capacity, 1, w.splits_max,
                          static_cast<cudaStream_t>(stream));
@@ -438,7 +449,7 @@ extern "C" int verify_attend_paged(const masw_paged_kv_desc* kv, const void* q, 
   const float scale = kv->softmax_scale > 0.f ? kv->softmax_scale : 1.0f / sqrtf(static_cast<float>(kv->head_dim));
   p.scale_log2e = scale * 1.4426950408889634f;
   if (T * G <= 32)
-    return launch_attend_tc<32, 3, 3>(tk, tv, p, kv->batch, kv->n_kv_heads, kv->max_pages, w.splits_max, static_cast<cudaStream_t>(stream));
-  return launch_attend_tc<64, 2, 3>(tk, tv, p, kv->batch, kv->n_kv_heads, kv->max_pages, w.splits_max, static_cast<cudaStream_t>(stream));
+    return launch_attend_tc<32, 3, 3>(tk, tv, tk, tv, p, kv->batch, kv->n_kv_heads, kv->max_pages, w.splits_max, static_cast<cudaStream_t>(stream));
+  return launch_attend_tc<64, 2, 3>(tk, tv, tk, tv, p, kv->batch, kv->n_kv_heads, kv->max_pages, w.splits_max, static_cast<cudaStream_t>(stream));
 }
 

@@ -63,6 +63,7 @@ struct AttendParams {
   int early;               // draft (attend_draft_kernel): the counters, slot_pos and this layer's K/V are not written by
                            // the launch's immediate predecessor in the stream, so they may be read before the wait
   int deterministic;       // verify (tcgen05 kernel): every tile assigned statically, results repeat bit for bit
+  int next_hint;           // verify (tcgen05 kernel): the second pair of tensor maps names the next call's cache (L2 hint)
 #ifdef MASW_TRACE
   long long* trace;        // developer build: per-CTA phase timestamps (null = off)
   int drop_tile;           // developer build: the copy of this CTA-local tile is armed but never issued (-1 = off),
@@ -165,7 +166,7 @@ __device__ __forceinline__ void rec_fetch_item(const unsigned long long* ml_rec,
 // lives on the device, so replaying the launch from a CUDA graph works.
 // Must be called by all NTHREADS threads of the CTA; `scratch` is shared memory of at least
 // NTHREADS * 24 + 8 * D + 64 bytes.
-template <int D, int KROWS, int NTHREADS>
+template <int D, int KROWS, int NTHREADS, int kGroups = 4, int kFetch = 6>
 __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, int b, int kvh, int split, int n_rows,
                                                        int epoch, float* scratch, int tid,
                                                        const double* rope_cs = nullptr, long long* tr = nullptr) {
@@ -180,8 +181,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
   const int per = (n_items + splits - 1) / splits;
   const int i_begin = split * per;
   const int my_items = max(0, min(n_items, i_begin + per) - i_begin);
-  constexpr int kGroups = 4;
-  constexpr int kSlots = NTHREADS / kGroups;
+  constexpr int kSlots = NTHREADS / kGroups;   // kGroups thread groups per item, each with kFetch splits' records in flight
   float* gsm = scratch;   // [kGroups][kSlots][6]: m, l, o4
   bool timed_out = false;
 
@@ -325,13 +325,13 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
     const float4 v_new = with_slot ? make_float4(vg[d4], vg[d4 + 1], vg[d4 + 2], vg[d4 + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
     const float* const my_gsm = gsm + (tid / kGroups) * 6;
     if (live) {
-      for (int sp0 = grp; sp0 < splits; sp0 += kGroups * 6) {
-        float2 ml[6];
-        float4 v[6];
-        bool okv[6];
+      for (int sp0 = grp; sp0 < splits; sp0 += kGroups * kFetch) {
+        float2 ml[kFetch];
+        float4 v[kFetch];
+        bool okv[kFetch];
         bool all_ok = true;
 #pragma unroll
-        for (int u = 0; u < 6; ++u) {
+        for (int u = 0; u < kFetch; ++u) {
           okv[u] = true;
           const int sp = sp0 + u * kGroups;
           if (sp < splits) {
@@ -344,7 +344,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
           __nanosleep(20);
           all_ok = true;
 #pragma unroll
-          for (int u = 0; u < 6; ++u) {
+          for (int u = 0; u < kFetch; ++u) {
             if (!okv[u]) {
               const int sp = sp0 + u * kGroups;
               rec_fetch_item(all_ml + (sp * KROWS + r) * 2, all_o + (static_cast<size_t>(sp) * KROWS + r) * D + d4, tag,
@@ -357,14 +357,14 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
         MASW_CLOCK(tr, 11);   // developer build: thread 0 holds every split's record of its first item
         float mb = m_run2;
 #pragma unroll
-        for (int u = 0; u < 6; ++u) if (sp0 + u * kGroups < splits) mb = fmaxf(mb, ml[u].x);
+        for (int u = 0; u < kFetch; ++u) if (sp0 + u * kGroups < splits) mb = fmaxf(mb, ml[u].x);
         const float mu = (mb == kNegInf) ? 0.f : mb;
         const float c = fast_exp2(m_run2 - mu);
         o4.x *= c; o4.y *= c; o4.z *= c; o4.w *= c;
         l_run2 *= c;
         m_run2 = mb;
 #pragma unroll
-        for (int u = 0; u < 6; ++u) {
+        for (int u = 0; u < kFetch; ++u) {
           if (sp0 + u * kGroups < splits) {
             const float w = fast_exp2(ml[u].x - mu);   // exp2(-inf) = 0 for an empty split
             o4.x += w * v[u].x; o4.y += w * v[u].y; o4.z += w * v[u].z; o4.w += w * v[u].w;
@@ -378,23 +378,21 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
     __syncthreads();
     MASW_CLOCK(tr, 12);     // developer build: every item of this CTA has all its records
     if (live && grp == 0) {
-      float2 part[kGroups][3];   // m, l | o.x, o.y | o.z, o.w of each group's partial
-#pragma unroll
-      for (int g2 = 0; g2 < kGroups; ++g2) {
-#pragma unroll
-        for (int k = 0; k < 3; ++k) part[g2][k] = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6 + 2 * k);
-      }
+      // the groups' partials (m, l | o.x, o.y | o.z, o.w), merged in group order
       float m = kNegInf;
 #pragma unroll
-      for (int g2 = 0; g2 < kGroups; ++g2) m = fmaxf(m, part[g2][0].x);
+      for (int g2 = 0; g2 < kGroups; ++g2) m = fmaxf(m, my_gsm[g2 * kSlots * 6]);
       if (with_slot) m = fmaxf(m, s_new);
       float l = 0.f;
       float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int g2 = 0; g2 < kGroups; ++g2) {
-        const float w = (part[g2][0].x == kNegInf) ? 0.f : fast_exp2(part[g2][0].x - m);
-        l += w * part[g2][0].y;
-        o.x += w * part[g2][1].x; o.y += w * part[g2][1].y; o.z += w * part[g2][2].x; o.w += w * part[g2][2].y;
+        const float2 ml2 = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6);
+        const float2 oa = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6 + 2);
+        const float2 ob = *reinterpret_cast<const float2*>(my_gsm + g2 * kSlots * 6 + 4);
+        const float w = (ml2.x == kNegInf) ? 0.f : fast_exp2(ml2.x - m);
+        l += w * ml2.y;
+        o.x += w * oa.x; o.y += w * oa.y; o.z += w * ob.x; o.w += w * ob.y;
       }
       if (with_slot) {
         const float w_new = fast_exp2(s_new - m);

@@ -167,7 +167,8 @@ static_assert(offsetof(TcCtrl<32>, bcast) % 16 == 0 && offsetof(TcCtrl<64>, bcas
 
 template <int NQ, int NK, int NV>
 __global__ void __launch_bounds__(TcCfg<NQ, NK, NV>::kThreads, 1)
-attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttendParams p) {
+attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                 const __grid_constant__ CUtensorMap tmKn, const __grid_constant__ CUtensorMap tmVn, const AttendParams p) {
   using C = TcCfg<NQ, NK, NV>;
   constexpr int D = 128;
   constexpr float kNegInf = -INFINITY;
@@ -193,6 +194,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   MASW_STAMP(tr, 0);
   // producer state (thread 0 only): the schedule and the pool claim in flight
   constexpr int kStaticNum = 1, kStaticDen = 4;   // share of the tiles that is assigned statically
+  constexpr int kHintStatic = 1;                  // statically assigned tiles per CTA named in the next call's L2 hint
   int n_static = 0, static_first = 0, n_pool = 0, n_early = 0, pending = 0x7fffffff;
   int* pool_ctr = nullptr;
   // ---- prologue
@@ -215,34 +217,60 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     mbar_init(&ctl->o_ready, 1);
     fence_mbar_init();
   }
-  // nothing above touched global memory: a launch that was allowed to start early waits here for its
+  // The CTA's first tile is tile number `split`, whatever the cache length turns out to be: it is requested
+  // before the length and the epoch have been loaded, which takes their round trip off the path to the first
+  // scores.  Should the cache be shorter than that, the tile is streamed all the same and fully masked.
+  // When the caller vouches that the kernel in front of this launch writes nothing of K and V (p.early), the
+  // request goes out before the wait: a CTA that starts while the predecessor's last CTAs are still draining
+  // then has its first tile on the way when the wait ends.
+  bool first_requested = false;
+  auto request_first_tile = [&]() {
+    const uint64_t policy = l2_policy_evict_first();
+    // contiguous cache: tile t of sequence b starts at entry 128 t; paged cache: it is page page_table[b][t]
+    // of the pool (the map's outermost coordinate), entries 0..127 of that page
+    int row0 = split * C::kTile, outer = b;
+    if (p.page_table != nullptr) {
+      outer = __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + split);
+      row0 = 0;
+      ctl->page_id[0] = outer;
+    }
+    mbar_arrive_expect_tx(&ctl->k_full[0], C::kTileBytes);
+    tma_load_4d(k_ring, &tmK, &ctl->k_full[0], 0, row0, kvh, outer, policy);
+    tma_load_4d(k_ring + C::kSubBytes, &tmK, &ctl->k_full[0], 64, row0, kvh, outer, policy);
+    mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
+    tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, row0, kvh, outer, policy);
+    tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, row0, kvh, outer, policy);
+    ctl->tile_id[0] = split;
+    n_early = 1;
+    first_requested = true;
+  };
+  if (tid == 0 && p.early && p.page_table == nullptr) request_first_tile();
+  // nothing else above touched global memory: a launch that was allowed to start early waits here for its
   // predecessor, and lets its own successor be set up
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (tid == 0) {
-    // The CTA's first tile is tile number `split`, whatever the cache length turns out to be: it is requested
-    // before the length and the epoch have been loaded, which takes their round trip off the path to the first
-    // scores.  Should the cache be shorter than that, the tile is streamed all the same and fully masked.
-    const uint64_t policy = l2_policy_evict_first();
-    {
-      // contiguous cache: tile t of sequence b starts at entry 128 t; paged cache: it is page page_table[b][t]
-      // of the pool (the map's outermost coordinate), entries 0..127 of that page
-      int row0 = split * C::kTile, outer = b;
-      if (p.page_table != nullptr) {
-        outer = __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + split);
-        row0 = 0;
-        ctl->page_id[0] = outer;
-      }
-      mbar_arrive_expect_tx(&ctl->k_full[0], C::kTileBytes);
-      tma_load_4d(k_ring, &tmK, &ctl->k_full[0], 0, row0, kvh, outer, policy);
-      tma_load_4d(k_ring + C::kSubBytes, &tmK, &ctl->k_full[0], 64, row0, kvh, outer, policy);
-      mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
-      tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, row0, kvh, outer, policy);
-      tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, row0, kvh, outer, policy);
-      ctl->tile_id[0] = split;
-      n_early = 1;
+  MASW_STAMP(tr, 10);
+  if (tid == 0 && !first_requested) request_first_tile();
+  // Everything this thread reads from global memory in the prologue is requested here, back to back, before any
+  // of it is used: the cache length, the reduction epoch and the thread's chunks of the Q tile then cost one
+  // round trip together instead of one each (thread 0 used to walk three dependent round trips).
+  constexpr int kChunksPerRow = D / 8;
+  constexpr int kQPerThread = (NQ * kChunksPerRow + C::kThreads - 1) / C::kThreads;
+  uint4 qv[kQPerThread];
+#pragma unroll
+  for (int k = 0; k < kQPerThread; ++k) {
+    const int idx = tid + k * C::kThreads;
+    const int r = idx / kChunksPerRow, cg = idx % kChunksPerRow;
+    qv[k] = make_uint4(0, 0, 0, 0);
+    if (idx < NQ * kChunksPerRow && r < n_rows) {
+      const int j = r / p.G, g = r % p.G;
+      qv[k] = __ldg(reinterpret_cast<const uint4*>(p.q + ((static_cast<size_t>(b) * p.n_q + j) * p.Hq + kvh * p.G + g) * D + cg * 8));
     }
-    const int len = min(max(p.kv_len[b], 0), p.capacity);
+  }
+  const int len_raw = (tid < NQ) ? __ldg(p.kv_len + b) : 0;
+  const int epoch_raw = (tid == 0) ? __ldcg(p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1)) : 0;
+  if (tid == 0) {
+    const int len = min(max(len_raw, 0), p.capacity);
     const int nt = (len + C::kTile - 1) / C::kTile;
     // Tile schedule of the tiles behind the first `splits` ones.  A quarter of them is assigned statically
     // (n_static consecutive tiles per split, at the end of the cache, so that the ragged and masked last tile
@@ -264,7 +292,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       n_pool = rest - n_static * p.splits;
       static_first = p.splits + n_pool + split * n_static;
     }
-    const int epoch = __ldcg(p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1));
+    const int epoch = epoch_raw;
     pool_ctr = p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + (epoch & 1);
     pending = (n_pool > 0) ? atomicAdd(pool_ctr, 1) : 0x7fffffff;   // used only after the static tiles
     ctl->plan[0] = len;
@@ -277,21 +305,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   }
   if (tid < NQ) {
     // row j of the T new tokens sees cache entries [0, len - T + j]; padding rows copy the last real row
-    const int len = min(max(p.kv_len[b], 0), p.capacity);
+    const int len = min(max(len_raw, 0), p.capacity);
     const int r = min(tid, n_rows - 1);
     ctl->row_lo[tid] = 0;
     ctl->row_hi[tid] = min(len - p.n_q + r / p.G, len - 1);
   }
-  {
-    constexpr int kChunksPerRow = D / 8;
-    for (int idx = tid; idx < NQ * kChunksPerRow; idx += C::kThreads) {
+#pragma unroll
+  for (int k = 0; k < kQPerThread; ++k) {
+    const int idx = tid + k * C::kThreads;
+    if (idx < NQ * kChunksPerRow) {
       const int r = idx / kChunksPerRow, cg = idx % kChunksPerRow;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (r < n_rows) {
-        const int j = r / p.G, g = r % p.G;
-        val = __ldg(reinterpret_cast<const uint4*>(p.q + ((static_cast<size_t>(b) * p.n_q + j) * p.Hq + kvh * p.G + g) * D + cg * 8));
-      }
-      *reinterpret_cast<uint4*>(q_smem + (cg >> 3) * C::kQSubBytes + r * 128 + (((cg & 7) ^ (r & 7)) << 4)) = val;
+      *reinterpret_cast<uint4*>(q_smem + (cg >> 3) * C::kQSubBytes + r * 128 + (((cg & 7) ^ (r & 7)) << 4)) = qv[k];
     }
   }
   fence_proxy_async();   // the Q tile was written with ordinary stores and is read by the tensor core
@@ -377,6 +401,24 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       }
       if (!k_done || !v_done) ctl->error = 1;
       ctl->plan[2] = iv;
+      // Every tile of this launch is requested: ask for the tile this CTA will stream first in the NEXT call (the
+      // next layer's cache, same geometry) to be brought into L2.  The requests queue behind this CTA's own last
+      // tiles and land while the launch is in its reduction, so the next launch's first tile is an L2 hit.
+      if (p.next_hint) {
+        tma_prefetch_4d(&tmKn, 0, split * C::kTile, kvh, b);
+        tma_prefetch_4d(&tmKn, 64, split * C::kTile, kvh, b);
+        tma_prefetch_4d(&tmVn, 0, split * C::kTile, kvh, b);
+        tma_prefetch_4d(&tmVn, 64, split * C::kTile, kvh, b);
+        // ... and its statically assigned tiles, which it streams next (the same numbers when the next cache is as
+        // long): HBM is idle while this launch publishes and reduces, and these bytes then need not cross it again
+        for (int i = 0; i < min(n_static, kHintStatic); ++i) {
+          const int row0 = (static_first + i) * C::kTile;
+          tma_prefetch_4d(&tmKn, 0, row0, kvh, b);
+          tma_prefetch_4d(&tmKn, 64, row0, kvh, b);
+          tma_prefetch_4d(&tmVn, 0, row0, kvh, b);
+          tma_prefetch_4d(&tmVn, 64, row0, kvh, b);
+        }
+      }
     }
   } else if (warp == 1) {
     // ================= MMA issuer =================
@@ -647,7 +689,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
   }
   MASW_STAMP(tr, 3);
-  split_reduce_and_store<D, NQ, C::kThreads>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
+  // six thread groups per item with three splits' records in flight each: 18 splits in one round trip, and few
+  // enough registers that nothing spills
+  split_reduce_and_store<D, NQ, C::kThreads, 6, 3>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
   // the pool counter of the next launch (the other parity) is idle now: clear it
   if (split == 0 && tid == 0) p.tickets[(b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + ((ctl->plan[6] + 1) & 1)] = 0;
   MASW_STAMP(tr, 4);
