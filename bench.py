@@ -37,6 +37,19 @@ SMI_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.acti
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
 
+def verify_hint_bytes(wl):
+    """Bytes of the next layer's cache a verify launch asks to be brought into L2 (masw_kv_desc.next_k / next_v): per
+    CTA tile number `split` and, where a CTA has statically assigned tiles, the first of them (128 entries each, K and
+    V).  Averaged over the layers of a step (the last layer has no successor)."""
+    heads = wl.batch * wl.t_kv_heads
+    splits = max(1, min(148 // heads, 64))
+    tiles = (wl.prefix + wl.gamma + 127) // 128
+    splits = min(splits, tiles)
+    n_static = (max(0, tiles - splits) // 4) // splits
+    per_cta = (1 + min(n_static, 1)) * 128 * wl.t_head_dim * 2 * 2
+    return splits * heads * per_cta * (wl.t_layers - 1) / wl.t_layers
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -646,9 +659,12 @@ def run_gpu(args, wl):
             "roofline": {"kernel": "attend_tc_kernel (verify_attend, one target layer per launch)", "bound": "hbm",
                          "achieved": v_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                          "frac": v_gbs / peak, "frac_of_8tbs": v_gbs / 8000.0,
-                         "traffic": args.traffic_bytes if args.traffic_bytes else verify_bytes_layer * NCU_TRAFFIC_RATIO,
-                         "traffic_source": "ncu dram bytes of an 8K-prefix launch (profiles/attend_kernels_cfg2_full.md) "
-                                           "scaled by KV bytes; traffic grows in proportion to the entries",
+                         "traffic": args.traffic_bytes if args.traffic_bytes
+                         else verify_bytes_layer * NCU_TRAFFIC_RATIO + verify_hint_bytes(wl),
+                         "traffic_source": "ncu dram bytes of an 8K-prefix launch (profiles/attend_kernels_cfg2_full.md): the "
+                                           "launch's own bytes scaled by KV bytes (x 1.014, traffic grows in proportion to the "
+                                           "entries) + the next layer's first tiles it asks into L2 (%.1f MB per launch, which "
+                                           "the next launch then does not read from DRAM)" % (verify_hint_bytes(wl) / 1e6),
                          "algorithmic_bytes_per_launch": verify_bytes_layer,
                          "launches_timed": wl.t_layers * K * n_blocks, "avg_launch_us": verify_us / wl.t_layers},
             # the other half of the step: the draft's decode launch (16.8 MB of KV per launch at batch 1, latency-bound)
