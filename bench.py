@@ -846,6 +846,70 @@ def run_prefill(args, wl):
     print(json.dumps(row), flush=True)
 
 
+def run_fp8(args):
+    """The verifier's attention over the paged cache in bf16 and in FP8 (e4m3 pages, one scale per page and KV head):
+    microseconds per target layer at 32K prefix on the 8B target shape for batch 1, 4 and 16, each timed as a CUDA
+    graph over several layers' pools (more bytes than L2).  One JSON line per batch size."""
+    import torch
+    from paper_2608_30252_b200 import build, binding
+    if not torch.cuda.is_available():
+        raise RuntimeError("the FP8 comparison needs a CUDA device")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    build.build()
+    binding.load()
+    peak, _ = measured_peak_gbs()
+    Hq, Hkv, D, P, T = 32, 8, 128, 32768, 5
+    for B in (1, 4, 16):
+        L = 4 if B < 16 else 2
+        max_pages = (P + T + 127) // 128
+        n_pages = B * max_pages
+        gen = torch.Generator(device=dev).manual_seed(260830252 + B)
+        table = torch.randperm(n_pages, device=dev, generator=gen).to(torch.int32).view(B, max_pages).contiguous()
+        kv_len = torch.full((B,), P + T, dtype=torch.int32, device=dev)
+        q = torch.randn((B, T, Hq, D), device=dev, generator=gen).to(torch.bfloat16)
+        o = torch.empty((B, T, Hq, D), dtype=torch.float32, device=dev)
+        lse = torch.empty((B, T, Hq), dtype=torch.float32, device=dev)
+        res = {}
+        for kind in ("bf16", "fp8"):
+            if kind == "bf16":
+                Ks = [torch.randn((n_pages, Hkv, 128, D), device=dev, generator=gen).to(torch.bfloat16) for _ in range(2 * L)]
+                call = lambda l, ws: binding.verify_attend_paged(Ks[2 * l], Ks[2 * l + 1], table, kv_len, q, workspace=ws, out=o, lse=lse)
+            else:   # random bytes below the NaN pattern stand in for quantised values: timing does not depend on them
+                Ks = [torch.randint(0, 0x7E, (n_pages, Hkv, 128, D), device=dev, dtype=torch.uint8, generator=gen) for _ in range(2 * L)]
+                sc = torch.full((n_pages, Hkv), 0.01, device=dev)
+                call = lambda l, ws: binding.verify_attend_fp8(Ks[2 * l], Ks[2 * l + 1], sc, sc, table, kv_len, q, workspace=ws, out=o, lse=lse)
+            ws = call(0, None)[2]
+            for l in range(L):
+                call(l, ws)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for l in range(L):
+                        call(l, ws)
+            torch.cuda.current_stream().wait_stream(side)
+            for _ in range(3):
+                g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            res[kind] = e0.elapsed_time(e1) * 1e3 / (10 * L)
+            del Ks
+            torch.cuda.empty_cache()
+        entries_bytes = 2 * (P + T) * Hkv * D * B
+        print(json.dumps({"metric": "verify attention us per target layer, paged cache, 32K prefix", "batch": B, "rows": T,
+                          "bf16_us": res["bf16"], "fp8_us": res["fp8"], "fp8_speedup": res["bf16"] / res["fp8"],
+                          "bf16_kv_gbs": entries_bytes * 2 / (res["bf16"] * 1e-6) / 1e9,
+                          "fp8_kv_gbs": entries_bytes / (res["fp8"] * 1e-6) / 1e9, "hbm_peak_gbs": peak,
+                          "cache_bytes_per_layer": {"bf16": entries_bytes * 2, "fp8": entries_bytes}}), flush=True)
+
+
 def run_loop(args):
     """The packaged speculative-decoding loop (paper_2608_30252_b200.loop) on its toy one-layer models: greedy
     decoding of 256 tokens after a 2000-token prompt, gamma = 5, draft memory S = 4, W = 256, r = 8.  Prints one JSON
@@ -1081,6 +1145,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the prefix x batch x gamma x ratio sweep (one JSON line per point)")
     ap.add_argument("--prefill", action="store_true",
                     help="time the draft's masked prefill pass (one layer per step) instead of the decoding iteration")
+    ap.add_argument("--fp8", action="store_true",
+                    help="verify attention over the paged cache in bf16 and in FP8 (e4m3): us per target layer at batch 1, 4, 16")
     ap.add_argument("--loop", action="store_true",
                     help="run the packaged speculative-decoding loop on its toy models: Tok./Iter, t_d, t_t, Eq. 1")
     ap.add_argument("--timeline", action="store_true",
@@ -1091,6 +1157,8 @@ def main():
     wl = inputs.WORKLOADS[args.workload]
     if args.sweep:
         run_sweep(args)
+    elif args.fp8:
+        run_fp8(args)
     elif args.loop:
         run_loop(args)
     elif args.timeline:

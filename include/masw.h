@@ -272,6 +272,36 @@ size_t verify_paged_workspace_bytes(const masw_paged_kv_desc* kv, int T);
 int verify_attend_paged(const masw_paged_kv_desc* kv, const void* q, int T, float* o, float* lse, void* o_bf16,
                         void* workspace /*[device]*/, size_t workspace_bytes, void* stream);
 
+/* An FP8 verifier cache (a serving variant beside the paged bf16 cache, Section 5.1: the target's KV bytes are what
+ * Eq. 2's beta L d term counts, and e4m3 halves them).  Pages of 128 entries, K and V laid out
+ * [page][kv head][128][head_dim] with ONE BYTE per element (e4m3: 1 sign, 4 exponent, 3 mantissa bits, bias 7, no
+ * infinities), and one fp32 scale per (page, kv head) for K and for V.  The value an element stands for is
+ * DEFINED as  fp16( e4m3_value x fp16(scale) )  (both roundings to nearest): the kernel forms exactly that product
+ * when it turns a page into an fp16 operand tile, and attention is then exact arithmetic on those values (q is
+ * rounded from bf16 to fp16 as well; probabilities go to the tensor cores as fp16). */
+typedef struct masw_fp8_kv_desc {
+  const void* k_pages;       /* [device] e4m3 bytes [n_pages][n_kv_heads][128][head_dim] */
+  const void* v_pages;       /* [device] same layout */
+  const float* k_scale;      /* [device] fp32 [n_pages][n_kv_heads] */
+  const float* v_scale;      /* [device] fp32 [n_pages][n_kv_heads] */
+  const int32_t* page_table; /* [device] [batch][max_pages]: pool page holding entries [128 i, 128 i + 128) of the sequence */
+  int32_t n_pages, max_pages;
+  int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128 */
+  const int32_t* kv_len;     /* [device] [batch] entries in use, INCLUDING the T rows being verified; <= 128 max_pages */
+  float softmax_scale;       /* 0 selects 1 / sqrt(D) */
+  int32_t flags;             /* MASW_KV_DETERMINISTIC or 0 */
+  int32_t* status;           /* [device] one int32 that receives MASW_STATUS_* bits (OR-ed in), or NULL */
+} masw_fp8_kv_desc;
+
+/* Scratch bytes for verify_attend_fp8 (same rules as verify_workspace_bytes).  Host only. */
+size_t verify_fp8_workspace_bytes(const masw_fp8_kv_desc* kv, int T);
+
+/* verify_attend (Section 4.3) over the FP8 paged cache: row j of the T new tokens attends causally to entries
+ * [0, kv_len[b] - T + j], each standing for its dequantised value as defined above.  q [device] bf16
+ * [batch][T][Hq][D]; outputs as in verify_attend.  T * (Hq/Hkv) must be <= 32. */
+int verify_attend_fp8(const masw_fp8_kv_desc* kv, const void* q, int T, float* o, float* lse, void* o_bf16,
+                      void* workspace /*[device]*/, size_t workspace_bytes, void* stream);
+
 /* Bytes of scratch accept_reject needs.  Host only.  Zero-fill once before first use. */
 size_t accept_workspace_bytes(int batch, int gamma, int vocab);
 

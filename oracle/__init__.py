@@ -19,3 +19,4 @@ from .verify import verify_attend  # noqa: F401
 from .prefill import prefill_attend, n_prefill_slots  # noqa: F401
 from .accept_reject import accept_reject, spec_exp, integer_weights  # noqa: F401
 from .speedup import sd_speedup, tokens_per_second  # noqa: F401
+from .fp8 import dequantize_e4m3, e4m3_to_f64, fp16_round  # noqa: F401

@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = [
     "masw_sizes", "mem_init", "mem_free", "mem_load", "mem_set_state", "mem_get_state", "mem_update",
     "mem_advance", "mem_rollback", "draft_attend", "draft_append_attend", "draft_boundary_attend", "draft_prefill_slots",
     "draft_prefill_attend", "verify_workspace_bytes", "verify_attend", "verify_paged_workspace_bytes", "verify_attend_paged",
+    "verify_fp8_workspace_bytes", "verify_attend_fp8",
     "accept_workspace_bytes", "accept_reject", "accept_reject_static", "masw_last_error", "masw_launch_count", "masw_version",
 ]
 
@@ -373,6 +374,47 @@ def verify_attend_paged(k_pages, v_pages, page_table, kv_len, q, workspace=None,
         lse = torch.empty((B, T, Hq), dtype=torch.float32, device=q.device)
     _check(lib.verify_attend_paged(C.byref(desc), _ptr(q), T, _ptr(out), _ptr(lse), _ptr(out_bf16), _ptr(workspace),
                                    workspace.numel(), _stream()))
+    return out, lse, workspace
+
+
+class masw_fp8_kv_desc(C.Structure):
+    _fields_ = [("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
+                ("page_table", C.c_void_p), ("n_pages", C.c_int32), ("max_pages", C.c_int32), ("batch", C.c_int32),
+                ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("kv_len", C.c_void_p),
+                ("softmax_scale", C.c_float), ("flags", C.c_int32), ("status", C.c_void_p)]
+
+
+def verify_attend_fp8(k_pages, v_pages, k_scale, v_scale, page_table, kv_len, q, workspace=None, out=None, lse=None,
+                      out_bf16=None, softmax_scale=0.0, deterministic=False, status=None):
+    """k_pages, v_pages: uint8 (e4m3 bytes) [n_pages, Hkv, 128, 128] contiguous; k_scale, v_scale fp32 [n_pages, Hkv];
+    page_table int32 [B, max_pages]; kv_len int32 [B] (including the T rows); q bf16 [B, T, Hq, 128].
+    Returns (o fp32, lse fp32, workspace)."""
+    assert k_pages.dtype == torch.uint8 and v_pages.dtype == torch.uint8 and k_pages.is_contiguous() and v_pages.is_contiguous()
+    assert k_pages.shape == v_pages.shape and k_scale.dtype == torch.float32 and v_scale.dtype == torch.float32
+    assert k_scale.is_contiguous() and v_scale.is_contiguous()
+    assert page_table.dtype == torch.int32 and page_table.is_contiguous() and kv_len.dtype == torch.int32
+    assert q.dtype == torch.bfloat16 and q.is_contiguous()
+    n_pages, Hkv, page, D = k_pages.shape
+    assert page == 128 and D == 128 and tuple(k_scale.shape) == (n_pages, Hkv) == tuple(v_scale.shape)
+    B, T, Hq, _ = q.shape
+    desc = masw_fp8_kv_desc(k_pages.data_ptr(), v_pages.data_ptr(), k_scale.data_ptr(), v_scale.data_ptr(),
+                            page_table.data_ptr(), n_pages, page_table.shape[1], B, Hq, Hkv, D, kv_len.data_ptr(),
+                            softmax_scale, KV_DETERMINISTIC if deterministic else 0,
+                            None if status is None else status.data_ptr())
+    lib = load()
+    lib.verify_fp8_workspace_bytes.argtypes = [C.POINTER(masw_fp8_kv_desc), C.c_int]
+    lib.verify_fp8_workspace_bytes.restype = C.c_size_t
+    lib.verify_attend_fp8.argtypes = [C.POINTER(masw_fp8_kv_desc), C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.verify_attend_fp8.restype = C.c_int
+    if workspace is None:
+        workspace = torch.zeros(lib.verify_fp8_workspace_bytes(C.byref(desc), T), dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty((B, T, Hq, D), dtype=torch.float32, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, T, Hq), dtype=torch.float32, device=q.device)
+    _check(lib.verify_attend_fp8(C.byref(desc), _ptr(q), T, _ptr(out), _ptr(lse), _ptr(out_bf16), _ptr(workspace),
+                                 workspace.numel(), _stream()))
     return out, lse, workspace
 
 

@@ -82,6 +82,22 @@ int encode_kv_tensor_map(CUtensorMap* out, const void* base, int head_dim, int64
   return MASW_OK;
 }
 
+// A pool of FP8 pages [page][kv head][128 entries][128 bytes] as a 4-D byte tensor (byte of the entry, entry of
+// the page, kv head, page) with a [128 x 128] box and 128-byte swizzle.
+int encode_fp8_page_map(CUtensorMap* out, const void* base, int n_kv_heads, int n_pages) {
+  EncodeTiledFn fn = encode_fn();
+  MASW_REQUIRE(fn != nullptr, MASW_ECUDA, "cuTensorMapEncodeTiled is unavailable (no CUDA driver?)");
+  cuuint64_t dims[4] = {128u, 128u, static_cast<cuuint64_t>(n_kv_heads), static_cast<cuuint64_t>(n_pages)};
+  cuuint64_t strides[3] = {128u, 128u * 128u, static_cast<cuuint64_t>(n_kv_heads) * 128u * 128u};
+  cuuint32_t box[4] = {128u, 128u, 1u, 1u};
+  cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, elem,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  MASW_REQUIRE(r == CUDA_SUCCESS, MASW_ECUDA, "cuTensorMapEncodeTiled (FP8 pages) failed with %d", static_cast<int>(r));
+  return MASW_OK;
+}
+
 }  // namespace masw
 
 extern "C" {

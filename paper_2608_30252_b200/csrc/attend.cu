@@ -108,11 +108,11 @@ static int launch_attend_draft(const CUtensorMap& tmK, const CUtensorMap& tmV, A
 }
 
 // tcgen05 / TMEM kernel (head_dim 128): query rows padded to NQ, rings of NK K tiles and NV V tiles (32 KB each)
-template <int NQ, int NK, int NV>
+template <int NQ, int NK, int NV, bool FP8 = false>
 static int launch_attend_tc(const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmKn, const CUtensorMap& tmVn,
                             AttendParams p, int B, int Hkv, int tiles_upper, int splits_max, cudaStream_t st) {
-  using C = TcCfg<NQ, NK, NV>;
-  auto kern = attend_tc_kernel<NQ, NK, NV>;
+  using C = TcCfg<NQ, NK, NV, FP8>;
+  auto kern = attend_tc_kernel<NQ, NK, NV, FP8>;
   static PerDeviceOnce once;
   { const int rc = set_smem_once(kern, C::kSmemBytes, once); if (rc != MASW_OK) return rc; }
   int splits = sm_count() / (B * Hkv);
@@ -453,3 +453,57 @@ extern "C" int verify_attend_paged(const masw_paged_kv_desc* kv, const void* q, 
   return launch_attend_tc<64, 2, 3>(tk, tv, tk, tv, p, kv->batch, kv->n_kv_heads, kv->max_pages, w.splits_max, static_cast<cudaStream_t>(stream));
 }
 
+
+// ---- verify_attend_fp8: the verifier's attention over a paged e4m3 cache ---------------------------------
+extern "C" size_t verify_fp8_workspace_bytes(const masw_fp8_kv_desc* kv, int T) {
+  if (kv == nullptr || T < 1 || kv->n_kv_heads < 1 || kv->n_q_heads % kv->n_kv_heads != 0) return 0;
+  return verify_ws(kv->batch, kv->n_kv_heads, kv->n_q_heads / kv->n_kv_heads, kv->head_dim, T).total;
+}
+
+extern "C" int verify_attend_fp8(const masw_fp8_kv_desc* kv, const void* q, int T, float* o, float* lse, void* o_bf16,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  MASW_REQUIRE(kv != nullptr && q != nullptr && o != nullptr && workspace != nullptr, MASW_EINVAL,
+               "verify_attend_fp8: null argument");
+  MASW_REQUIRE(kv->k_pages != nullptr && kv->v_pages != nullptr && kv->k_scale != nullptr && kv->v_scale != nullptr &&
+                   kv->page_table != nullptr && kv->kv_len != nullptr,
+               MASW_EINVAL, "verify_attend_fp8: null cache pointer");
+  MASW_REQUIRE(kv->head_dim == 128, MASW_EINVAL, "verify_attend_fp8: head_dim must be 128");
+  MASW_REQUIRE(kv->batch >= 1 && kv->n_kv_heads >= 1 && kv->n_q_heads >= kv->n_kv_heads &&
+                   kv->n_q_heads % kv->n_kv_heads == 0 && kv->n_pages >= 1 && kv->max_pages >= 1,
+               MASW_EINVAL, "verify_attend_fp8: bad cache geometry");
+  const int G = kv->n_q_heads / kv->n_kv_heads;
+  MASW_REQUIRE(T >= 1 && T * G <= 32, MASW_EINVAL, "verify_attend_fp8: T * group size = %d exceeds 32", T * G);
+  MASW_REQUIRE(aligned16(kv->k_pages) && aligned16(kv->v_pages) && aligned16(q) && aligned16(o) && aligned16(o_bf16) &&
+                   aligned16(workspace),
+               MASW_EALIGN, "verify_attend_fp8: pointers must be 16-byte aligned");
+  const VerifyWs w = verify_ws(kv->batch, kv->n_kv_heads, G, kv->head_dim, T);
+  MASW_REQUIRE(workspace_bytes >= w.total, MASW_ECAPACITY, "verify_attend_fp8: workspace %zu < %zu bytes", workspace_bytes,
+               w.total);
+  CUtensorMap tk, tv;
+  int rc = encode_fp8_page_map(&tk, kv->k_pages, kv->n_kv_heads, kv->n_pages);
+  if (rc != MASW_OK) return rc;
+  rc = encode_fp8_page_map(&tv, kv->v_pages, kv->n_kv_heads, kv->n_pages);
+  if (rc != MASW_OK) return rc;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  AttendParams p{};
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.o = o; p.lse = lse; p.o_bf16 = static_cast<__nv_bfloat16*>(o_bf16);
+  p.part_o = reinterpret_cast<unsigned long long*>(ws + w.off_part_o);
+  p.part_ml = reinterpret_cast<unsigned long long*>(ws + w.off_part_ml);
+  p.tickets = reinterpret_cast<int*>(ws + w.off_tickets);
+  p.status = kv->status;
+  p.deterministic = (kv->flags & MASW_KV_DETERMINISTIC) ? 1 : 0;
+  p.kv_len = kv->kv_len;
+  p.n_q = T; p.last_row_is_slot = 0;
+  p.G = G; p.Hq = kv->n_q_heads; p.Hkv = kv->n_kv_heads;
+  p.S = 0; p.W = 0; p.ring_cap = 1; p.max_slots = 0;
+  p.capacity = kv->max_pages * 128;
+  p.page_table = kv->page_table;
+  p.max_pages = kv->max_pages;
+  p.k_scale = kv->k_scale; p.v_scale = kv->v_scale;
+  const float scale = kv->softmax_scale > 0.f ? kv->softmax_scale : 1.0f / sqrtf(static_cast<float>(kv->head_dim));
+  p.scale_log2e = scale * 1.4426950408889634f;
+  // one K operand buffer (free again as soon as S^T is computed), two V operand buffers, three raw tiles per ring
+  return launch_attend_tc<32, 1, 2, true>(tk, tv, tk, tv, p, kv->batch, kv->n_kv_heads, kv->max_pages, w.splits_max,
+                                          static_cast<cudaStream_t>(stream));
+}

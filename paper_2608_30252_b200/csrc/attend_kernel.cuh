@@ -56,6 +56,8 @@ struct AttendParams {
   int S, W, ring_cap, max_slots;
   int capacity;            // entries per (sequence, head) in the tensor map (paged: logical entries per sequence)
   const int* page_table;   // paged verifier cache: [B][max_pages] physical page of each 128-entry logical page, else null
+  const float* k_scale;    // FP8 verifier cache: [n_pages][Hkv] fp32 scale of each page's K (V) bytes, else null
+  const float* v_scale;
   int max_pages;
   int splits;
   float scale_log2e;

@@ -65,9 +65,9 @@ __device__ __forceinline__ uint64_t tc_desc_mnmajor_sw64(uint32_t saddr) {
   return static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(512 >> 4) << 16) |
          (static_cast<uint64_t>(512 >> 4) << 32) | (1ull << 46) | (4ull << 61);
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, M x N tile, operand majorness.
-__host__ __device__ constexpr uint32_t tc_idesc(int M, int N, int a_mn_major, int b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn_major) << 15) |
+// Instruction descriptor: fp32 accumulator, bf16 (or, with `f16`, fp16) A and B, M x N tile, operand majorness.
+__host__ __device__ constexpr uint32_t tc_idesc(int M, int N, int a_mn_major, int b_mn_major, bool f16 = false) {
+  return (1u << 4) | (f16 ? 0u : (1u << 7) | (1u << 10)) | (static_cast<uint32_t>(a_mn_major) << 15) |
          (static_cast<uint32_t>(b_mn_major) << 16) | (static_cast<uint32_t>(N >> 3) << 17) |
          (static_cast<uint32_t>(M >> 4) << 24);
 }
@@ -95,6 +95,33 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const float (&v)[16]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// two e4m3 values (the low 16 bits of `pair`) -> two fp16 values (exact: e4m3 is a subset of fp16)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t pair) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(d) : "h"(static_cast<unsigned short>(pair)));
+  return d;
+}
+__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {   // fp16x2 product, rounded to nearest
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ float f16_lo_to_f32(uint32_t v) {
+  float f;
+  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tcvt.f32.f16 %0, l;\n\t}" : "=f"(f) : "r"(v));
+  return f;
+}
+__device__ __forceinline__ float f16_hi_to_f32(uint32_t v) {
+  float f;
+  asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tcvt.f32.f16 %0, h;\n\t}" : "=f"(f) : "r"(v));
+  return f;
+}
 
 __device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
@@ -124,22 +151,29 @@ __device__ __forceinline__ float warp_transpose_reduce(float (&v)[N], int lane) 
   return r;
 }
 
-template <int NQ, int NK, int NV>
+// FP8: the cache holds e4m3 bytes (paged, one scale per page and KV head).  Raw 16 KB tiles stream into two small
+// rings; two otherwise idle warps turn each into the fp16 operand tile (same swizzled layout a bf16 tile has), and
+// every MMA runs on fp16 operands (Q converted on load, P written as fp16).  NK / NV then count operand buffers.
+template <int NQ, int NK, int NV, bool FP8 = false>
 struct TcCfg {
   static constexpr int D = 128;
   static constexpr int kTile = 128;                    // entries per KV tile
   static constexpr int kSoftGroups = 2;                // softmax groups of four warps, each owning half of the query rows
   static constexpr int kCols = NQ / kSoftGroups;       // query rows (TMEM columns) per group
-  static constexpr int kThreads = (4 + 4 * kSoftGroups) * 32;
+  static constexpr int kDeqWarps = 6;                  // FP8: warps 2, 3 and four more behind the softmax warps convert raw tiles
+  static constexpr int kThreads = (4 + 4 * kSoftGroups + (FP8 ? 4 : 0)) * 32;
   static constexpr int kSubBytes = kTile * 128;        // one [128 x 64] bf16 box
   static constexpr int kTileBytes = 2 * kSubBytes;     // K or V tile
   static constexpr int kKRingBytes = NK * kTileBytes;   // K tiles are released as soon as S^T is computed,
   static constexpr int kVRingBytes = NV * kTileBytes;   // V tiles only after P.V: two rings of their own depth
-  static constexpr int kPipeBytes = kKRingBytes + kVRingBytes;
+  static constexpr int kRawTileBytes = kTile * D;      // FP8: one [128 entries x 128 bytes] box
+  static constexpr int kRaw = 3;                        // FP8: raw tiles in flight per ring
+  static constexpr int kRawBytes = FP8 ? 2 * kRaw * kRawTileBytes : 0;
+  static constexpr int kPipeBytes = kKRingBytes + kVRingBytes + kRawBytes;
   static constexpr int kQSubBytes = NQ * 128;
   static constexpr int kQBytes = 2 * kQSubBytes;       // Q tile; the P tile has the same shape
   static constexpr int kTmemCols = (3 * NQ <= 128) ? 128 : 256;   // 2 x S^T + O^T, power of two
-  static constexpr int kCtrlBytes = 1536 + 4 * NQ * 4 * 5;
+  static constexpr int kCtrlBytes = 1792 + 4 * NQ * 4 * 5;
   static constexpr int kSmemBytes = 1024 + kPipeBytes + 3 * kQBytes + kCtrlBytes;   // Q tile + two P tiles
   static_assert(NQ == 32 || NQ == 64, "query rows padded to 32 or 64");
   static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -148,6 +182,7 @@ struct TcCfg {
 template <int NQ>
 struct TcCtrl {
   uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4], s_full[2], s_empty[2], p_full[2], p_empty[2], o_ready;
+  uint64_t k8_full[4], k8_empty[4], v8_full[4], v8_empty[4];   // FP8: the raw rings
   uint32_t tmem_base;
   int error;
   int plan[8];               // [0] cache length, [1] first static tile, [2] tiles this CTA streamed, [6] reduction epoch
@@ -165,12 +200,13 @@ static_assert(sizeof(TcCtrl<32>) <= TcCfg<32, 3, 3>::kCtrlBytes && sizeof(TcCtrl
               "control block must fit its shared-memory share");
 static_assert(offsetof(TcCtrl<32>, bcast) % 16 == 0 && offsetof(TcCtrl<64>, bcast) % 16 == 0, "bcast is read as float4");
 
-template <int NQ, int NK, int NV>
-__global__ void __launch_bounds__(TcCfg<NQ, NK, NV>::kThreads, 1)
+template <int NQ, int NK, int NV, bool FP8 = false>
+__global__ void __launch_bounds__(TcCfg<NQ, NK, NV, FP8>::kThreads, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmKn, const __grid_constant__ CUtensorMap tmVn, const AttendParams p) {
-  using C = TcCfg<NQ, NK, NV>;
+  using C = TcCfg<NQ, NK, NV, FP8>;
   constexpr int D = 128;
+  constexpr int kDeq = C::kDeqWarps;   // FP8: converting warps; an operand tile is complete when all have arrived
   constexpr float kNegInf = -INFINITY;
 
   extern __shared__ uint8_t smem_raw[];
@@ -178,6 +214,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   uint8_t* pipe = smem;                       // K ring, then V ring
   uint8_t* k_ring = smem;
   uint8_t* v_ring = smem + C::kKRingBytes;
+  uint8_t* k8_ring = smem + C::kKRingBytes + C::kVRingBytes;        // FP8 only
+  uint8_t* v8_ring = k8_ring + C::kRaw * C::kRawTileBytes;
   uint8_t* q_smem = smem + C::kPipeBytes;
   uint8_t* p_smem = q_smem + C::kQBytes;
   TcCtrl<NQ>* ctl = reinterpret_cast<TcCtrl<NQ>*>(p_smem + 2 * C::kQBytes);
@@ -210,8 +248,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // thread 0 is the TMA producer: it initialises the barriers, plans this CTA's tile range and puts
     // the first ring of tiles in flight before the CTA-wide barrier, so that the first HBM round trip
     // overlaps the rest of the prologue (Q tile, TMEM allocation)
-    for (int s = 0; s < NK; ++s) { mbar_init(&ctl->k_full[s], 1); mbar_init(&ctl->k_empty[s], 1); }
-    for (int s = 0; s < NV; ++s) { mbar_init(&ctl->v_full[s], 1); mbar_init(&ctl->v_empty[s], 1); }
+    // an operand tile is complete when TMA has delivered it, or (FP8) when both converting warps have written their half
+    for (int s = 0; s < NK; ++s) { mbar_init(&ctl->k_full[s], FP8 ? kDeq : 1); mbar_init(&ctl->k_empty[s], 1); }
+    for (int s = 0; s < NV; ++s) { mbar_init(&ctl->v_full[s], FP8 ? kDeq : 1); mbar_init(&ctl->v_empty[s], 1); }
+    if (FP8) {
+      for (int s = 0; s < C::kRaw; ++s) {
+        mbar_init(&ctl->k8_full[s], 1); mbar_init(&ctl->k8_empty[s], kDeq);
+        mbar_init(&ctl->v8_full[s], 1); mbar_init(&ctl->v8_empty[s], kDeq);
+      }
+    }
     for (int s = 0; s < 2; ++s) { mbar_init(&ctl->s_full[s], 1); mbar_init(&ctl->s_empty[s], 128 * C::kSoftGroups); }
     for (int s = 0; s < 2; ++s) { mbar_init(&ctl->p_full[s], 128 * C::kSoftGroups); mbar_init(&ctl->p_empty[s], 1); }
     mbar_init(&ctl->o_ready, 1);
@@ -234,12 +279,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       row0 = 0;
       ctl->page_id[0] = outer;
     }
-    mbar_arrive_expect_tx(&ctl->k_full[0], C::kTileBytes);
-    tma_load_4d(k_ring, &tmK, &ctl->k_full[0], 0, row0, kvh, outer, policy);
-    tma_load_4d(k_ring + C::kSubBytes, &tmK, &ctl->k_full[0], 64, row0, kvh, outer, policy);
-    mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
-    tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, row0, kvh, outer, policy);
-    tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, row0, kvh, outer, policy);
+    if (FP8) {
+      mbar_arrive_expect_tx(&ctl->k8_full[0], C::kRawTileBytes);
+      tma_load_4d(k8_ring, &tmK, &ctl->k8_full[0], 0, row0, kvh, outer, policy);
+      mbar_arrive_expect_tx(&ctl->v8_full[0], C::kRawTileBytes);
+      tma_load_4d(v8_ring, &tmV, &ctl->v8_full[0], 0, row0, kvh, outer, policy);
+    } else {
+      mbar_arrive_expect_tx(&ctl->k_full[0], C::kTileBytes);
+      tma_load_4d(k_ring, &tmK, &ctl->k_full[0], 0, row0, kvh, outer, policy);
+      tma_load_4d(k_ring + C::kSubBytes, &tmK, &ctl->k_full[0], 64, row0, kvh, outer, policy);
+      mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
+      tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, row0, kvh, outer, policy);
+      tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, row0, kvh, outer, policy);
+    }
     ctl->tile_id[0] = split;
     n_early = 1;
     first_requested = true;
@@ -315,6 +367,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int idx = tid + k * C::kThreads;
     if (idx < NQ * kChunksPerRow) {
       const int r = idx / kChunksPerRow, cg = idx % kChunksPerRow;
+      if (FP8) {   // the MMAs run on fp16 operands: q is rounded from bf16 to fp16 (exact but for values below 2^-14)
+        uint32_t* w = reinterpret_cast<uint32_t*>(&qv[k]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) w[e] = pack_f16x2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
+      }
       *reinterpret_cast<uint4*>(q_smem + (cg >> 3) * C::kQSubBytes + r * 128 + (((cg & 7) ^ (r & 7)) << 4)) = qv[k];
     }
   }
@@ -360,38 +417,52 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       int idle = 0;
       while ((!k_done || !v_done) && idle < MASW_WAIT_LIMIT(p)) {
         bool progressed = false;
-        if (!k_done && (ik < NK || mbar_try_wait(&ctl->k_empty[ik % NK], (ik / NK - 1) & 1))) {
+        // (FP8: the producer fills the raw rings; the converting warps fill the operand buffers from them)
+        constexpr int RK = FP8 ? C::kRaw : NK, RV = FP8 ? C::kRaw : NV;
+        uint64_t* const kf = FP8 ? ctl->k8_full : ctl->k_full;
+        uint64_t* const ke = FP8 ? ctl->k8_empty : ctl->k_empty;
+        uint64_t* const vf = FP8 ? ctl->v8_full : ctl->v_full;
+        uint64_t* const ve = FP8 ? ctl->v8_empty : ctl->v_empty;
+        if (!k_done && (ik < RK || mbar_try_wait(&ke[ik % RK], (ik / RK - 1) & 1))) {
           const int id = resolve(ik);
           if (id < 0) {
-            mbar_arrive(&ctl->k_full[ik % NK]);
+            mbar_arrive(&kf[ik % RK]);
             k_done = true;
           } else {
-            uint8_t* kdst = k_ring + (ik % NK) * C::kTileBytes;
             const bool paged = p.page_table != nullptr;
             const int row0 = paged ? 0 : id * C::kTile, outer = paged ? ctl->page_id[ik & 15] : b;
-            mbar_arrive_expect_tx(&ctl->k_full[ik % NK], C::kTileBytes);
+            mbar_arrive_expect_tx(&kf[ik % RK], FP8 ? C::kRawTileBytes : C::kTileBytes);
 #ifdef MASW_TRACE
             if (ik != p.drop_tile)
 #endif
             {
-              tma_load_4d(kdst, &tmK, &ctl->k_full[ik % NK], 0, row0, kvh, outer, policy);
-              tma_load_4d(kdst + C::kSubBytes, &tmK, &ctl->k_full[ik % NK], 64, row0, kvh, outer, policy);
+              if (FP8) {
+                tma_load_4d(k8_ring + (ik % RK) * C::kRawTileBytes, &tmK, &kf[ik % RK], 0, row0, kvh, outer, policy);
+              } else {
+                uint8_t* kdst = k_ring + (ik % NK) * C::kTileBytes;
+                tma_load_4d(kdst, &tmK, &kf[ik % RK], 0, row0, kvh, outer, policy);
+                tma_load_4d(kdst + C::kSubBytes, &tmK, &kf[ik % RK], 64, row0, kvh, outer, policy);
+              }
             }
             ++ik;
           }
           progressed = true;
         }
-        if (!v_done && (iv < NV || mbar_try_wait(&ctl->v_empty[iv % NV], (iv / NV - 1) & 1))) {
+        if (!v_done && (iv < RV || mbar_try_wait(&ve[iv % RV], (iv / RV - 1) & 1))) {
           const int id = resolve(iv);
           if (id < 0) {
             v_done = true;
           } else {
-            uint8_t* vdst = v_ring + (iv % NV) * C::kTileBytes;
             const bool paged = p.page_table != nullptr;
             const int row0 = paged ? 0 : id * C::kTile, outer = paged ? ctl->page_id[iv & 15] : b;
-            mbar_arrive_expect_tx(&ctl->v_full[iv % NV], C::kTileBytes);
-            tma_load_4d(vdst, &tmV, &ctl->v_full[iv % NV], 0, row0, kvh, outer, policy);
-            tma_load_4d(vdst + C::kSubBytes, &tmV, &ctl->v_full[iv % NV], 64, row0, kvh, outer, policy);
+            mbar_arrive_expect_tx(&vf[iv % RV], FP8 ? C::kRawTileBytes : C::kTileBytes);
+            if (FP8) {
+              tma_load_4d(v8_ring + (iv % RV) * C::kRawTileBytes, &tmV, &vf[iv % RV], 0, row0, kvh, outer, policy);
+            } else {
+              uint8_t* vdst = v_ring + (iv % NV) * C::kTileBytes;
+              tma_load_4d(vdst, &tmV, &vf[iv % RV], 0, row0, kvh, outer, policy);
+              tma_load_4d(vdst + C::kSubBytes, &tmV, &vf[iv % RV], 64, row0, kvh, outer, policy);
+            }
             ++iv;
           }
           progressed = true;
@@ -423,11 +494,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   } else if (warp == 1) {
     // ================= MMA issuer =================
     if (lane == 0) {
-      constexpr uint32_t idesc1 = tc_idesc(128, NQ, 0, 0);   // K (K-major) x Q (K-major)
+      constexpr uint32_t idesc1 = tc_idesc(128, NQ, 0, 0, FP8);   // K (K-major) x Q (K-major)
       // V^T (MN-major) x P (MN-major too: [entry][row], one line of NQ rows per entry, 128 bytes with the 128B
       // swizzle or 64 bytes with the 64B swizzle, so that a softmax thread, which owns an entry, writes its
       // probabilities as 16-byte chunks of its own line)
-      constexpr uint32_t idesc2 = tc_idesc(128, NQ, 1, 1);
+      constexpr uint32_t idesc2 = tc_idesc(128, NQ, 1, 1, FP8);
       const uint32_t q_base = smem_u32(q_smem), p_base = smem_u32(p_smem);
       bool ok = true;
       int n_end = 0x7fffffff;   // index of the end-of-stream marker, once met
@@ -475,7 +546,67 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       }
       if (!ok) ctl->error = 1;
     }
-  } else if (warp >= 4) {
+  } else if (FP8 && (warp == 2 || warp == 3 || warp >= 12)) {
+    // ================= FP8: raw tile -> fp16 operand tile =================
+    // Six warps share every K and V tile (groups of four entries, dealt round-robin).  A lane takes one 16-byte chunk
+    // (16 e4m3 values of one entry), widens it to fp16 (exact), multiplies by the page's scale in fp16 (one
+    // rounding: this product IS the dequantised value the result is defined on) and writes the two 16-byte chunks
+    // into the operand tile in the swizzled layout a bf16 tile has.  The end of the stream travels on as it does
+    // for the bf16 cache: the producer completes the raw K barrier of an empty "tile", and the warps pass it to
+    // the MMA issuer through the operand barrier.
+    const int didx = warp < 4 ? warp - 2 : warp - 10;   // 0..5: takes every sixth group of four rows
+    const int c = lane & 7;                       // 16-byte chunk of the raw row: dims 16 c .. 16 c + 15
+    const int r_in = lane >> 3;                   // row inside a group of four
+    bool ok = true;
+    auto convert = [&](const uint8_t* raw, uint8_t* dst, uint32_t scale2) {
+#ifdef MASW_TRACE
+      if (p.debug_flags & 32) return;   // timing experiment: no conversion (results are then meaningless)
+#endif
+#pragma unroll 3
+      for (int it = didx; it < 32; it += kDeq) {
+        const int r = it * 4 + r_in;
+        const uint4 x = *reinterpret_cast<const uint4*>(raw + r * 128 + ((c ^ (r & 7)) << 4));
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+        uint32_t h[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          h[2 * e] = hmul2_u32(e4m3x2_to_f16x2(w[e] & 0xffffu), scale2);
+          h[2 * e + 1] = hmul2_u32(e4m3x2_to_f16x2(w[e] >> 16), scale2);
+        }
+        uint8_t* row = dst + (c >> 2) * C::kSubBytes + r * 128;
+        const int c16 = (c & 3) * 2;
+        *reinterpret_cast<uint4*>(row + (((c16) ^ (r & 7)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4*>(row + (((c16 + 1) ^ (r & 7)) << 4)) = make_uint4(h[4], h[5], h[6], h[7]);
+      }
+    };
+    for (int i = 0; ok; ++i) {
+      ok = mbar_wait_bounded(&ctl->k8_full[i % C::kRaw], (i / C::kRaw) & 1, MASW_WAIT_LIMIT(p));
+      if (!ok) break;
+      const int tile = ctl->tile_id[i & 15];
+      if (tile < 0) {   // end of the stream: hand it on to the MMA issuer
+        if (i >= NK) ok = mbar_wait_bounded(&ctl->k_empty[i % NK], (i / NK - 1) & 1, MASW_WAIT_LIMIT(p));
+        if (lane == 0) mbar_arrive(&ctl->k_full[i % NK]);
+        break;
+      }
+      const int page = ctl->page_id[i & 15];
+      const float ks = __ldg(p.k_scale + static_cast<size_t>(page) * p.Hkv + kvh);
+      const float vs = __ldg(p.v_scale + static_cast<size_t>(page) * p.Hkv + kvh);
+      if (i >= NK) ok = mbar_wait_bounded(&ctl->k_empty[i % NK], (i / NK - 1) & 1, MASW_WAIT_LIMIT(p));
+      if (!ok) break;
+      convert(k8_ring + (i % C::kRaw) * C::kRawTileBytes, k_ring + (i % NK) * C::kTileBytes, pack_f16x2(ks, ks));
+      fence_proxy_async();   // the operand tile was written with ordinary stores and is read by the tensor core
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&ctl->k_full[i % NK]); mbar_arrive(&ctl->k8_empty[i % C::kRaw]); }
+      ok = mbar_wait_bounded(&ctl->v8_full[i % C::kRaw], (i / C::kRaw) & 1, MASW_WAIT_LIMIT(p));
+      if (ok && i >= NV) ok = mbar_wait_bounded(&ctl->v_empty[i % NV], (i / NV - 1) & 1, MASW_WAIT_LIMIT(p));
+      if (!ok) break;
+      convert(v8_ring + (i % C::kRaw) * C::kRawTileBytes, v_ring + (i % NV) * C::kTileBytes, pack_f16x2(vs, vs));
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&ctl->v_full[i % NV]); mbar_arrive(&ctl->v8_empty[i % C::kRaw]); }
+    }
+    if (!ok) ctl->error = 1;
+  } else if (warp >= 4 && warp < 12) {
     // ================= softmax warps =================
     // kSoftGroups groups of four warps; group g owns the query rows (TMEM columns) [kCols g, kCols g + kCols), and
     // inside a group thread <-> TMEM lane <-> entry.  Columns are independent, so the groups only share the
@@ -575,10 +706,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         for (int k = 0; k < 4; k += 2) {   // two probabilities per conversion instruction
           const float pv0 = fast_exp2(fmaf(s[c4 + k], p.scale_log2e, nmu[k]));
           const float pv1 = fast_exp2(fmaf(s[c4 + k + 1], p.scale_log2e, nmu[k + 1]));
-          const uint32_t pr2 = pack_bf16x2(pv0, pv1);
+          const uint32_t pr2 = FP8 ? pack_f16x2(pv0, pv1) : pack_bf16x2(pv0, pv1);
           pk[(c4 + k) >> 1] = pr2;
-          l_part[c4 + k] = l_part[c4 + k] * cr[k] + __uint_as_float(pr2 << 16);
-          l_part[c4 + k + 1] = l_part[c4 + k + 1] * cr[k + 1] + __uint_as_float(pr2 & 0xffff0000u);
+          l_part[c4 + k] = l_part[c4 + k] * cr[k] + (FP8 ? f16_lo_to_f32(pr2) : __uint_as_float(pr2 << 16));
+          l_part[c4 + k + 1] = l_part[c4 + k + 1] * cr[k + 1] + (FP8 ? f16_hi_to_f32(pr2) : __uint_as_float(pr2 & 0xffff0000u));
         }
       }
 
@@ -691,7 +822,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   MASW_STAMP(tr, 3);
   // six thread groups per item with three splits' records in flight each: 18 splits in one round trip, and few
   // enough registers that nothing spills
-  split_reduce_and_store<D, NQ, C::kThreads, 6, 3>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
+  static_assert(C::kThreads % (FP8 ? 8 : 6) == 0, "the fetch groups must divide the thread count");
+  split_reduce_and_store<D, NQ, C::kThreads, FP8 ? 8 : 6, 3>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
   // the pool counter of the next launch (the other parity) is idle now: clear it
   if (split == 0 && tid == 0) p.tickets[(b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + ((ctl->plan[6] + 1) & 1)] = 0;
   MASW_STAMP(tr, 4);

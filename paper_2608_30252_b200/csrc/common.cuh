@@ -60,6 +60,9 @@ int encode_kv_tensor_map(CUtensorMap* out, const void* base, int head_dim, int64
 // the description (encoding costs a few microseconds of host time).
 int get_kv_maps(const masw_kv_desc& kv, int box_rows, CUtensorMap* tk, CUtensorMap* tv);
 
+// Tensor map of a pool of FP8 pages ([page][kv head][128][128] bytes), box = one page of one head.
+int encode_fp8_page_map(CUtensorMap* out, const void* base, int n_kv_heads, int n_pages);
+
 // ------------------------------------------------------------------------------------------------
 // device-side primitives
 #ifdef __CUDACC__

@@ -43,6 +43,19 @@ def uniforms_24bit(rng: np.random.Generator, shape) -> np.ndarray:
     return (k.astype(np.float64) * 2.0 ** -24).astype(np.float32)
 
 
+def quantize_e4m3_pages(x: np.ndarray):
+    """Quantises a float32 cache [n_pages, Hkv, 128, D] to e4m3 bytes with one scale per (page, KV head): scale =
+    amax / 448 (rounded to fp16, the precision the library uses it in), byte = nearest e4m3 of x / scale.  How a
+    serving stack quantises its cache is its own business; this is merely how the synthetic FP8 caches of the tests
+    and the benchmark are made.  Returns (uint8 bytes, float32 scales [n_pages, Hkv])."""
+    import torch
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    amax = np.abs(x).max(axis=(2, 3))
+    scale = np.maximum(amax / 448.0, 2.0 ** -14).astype(np.float16).astype(np.float32)
+    q = torch.from_numpy(x / scale[:, :, None, None]).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn)
+    return q.view(torch.uint8).numpy().copy(), scale
+
+
 def rng_for(config_id: int, layer: int = 0, stream: int = 0) -> np.random.Generator:
     """Seed recipe: base + 1000 * config + layer, with an extra stream index for independent draws."""
     return np.random.default_rng([BASE_SEED + 1000 * config_id + layer, stream])
