@@ -248,6 +248,56 @@ def test_full_size_memory_in_bench_launch_configuration(name, fused):
     _loaded_case(wl, layer_count=3, layer=2, rng=inputs.rng_for(wl.config_id, 2, 5), fused=fused)
 
 
+@pytest.mark.parametrize("name", ["cfg3_8b_32k", "cfg4_70b_32k"])
+def test_full_size_boundary_launches_ahead_of_their_predecessor(name):
+    """The benchmark's boundary launch at full size: draft_boundary_attend on consecutive layers, so that every launch
+    but the first runs ahead of its predecessor (plan, K/V copies, first tile in registers and the projection's weight
+    rows before the wait; 18 k-splits of the slot projection).  Each layer's two rows and its stored slot are checked
+    against the oracle."""
+    wl = inputs.WORKLOADS[name]
+    rng = inputs.rng_for(wl.config_id, 3, 6)
+    B, Hq, Hkv, D, S, M, W = wl.batch, wl.d_q_heads, wl.d_kv_heads, wl.d_head_dim, wl.sink, wl.slots, wl.window
+    L, d = 3, wl.d_model
+    cfg = binding.MaswConfig(L, B, Hq, Hkv, D, d, S, W, wl.slot_interval, rollback=16, max_slots=M + 8, gamma_max=8)
+    g = binding.DraftMemory(cfg)
+    t0 = S + M * wl.slot_interval
+    data = []
+    for l in range(L):
+        ks, vs = inputs.normal_bf16(rng, (B, M, Hkv, D)), inputs.normal_bf16(rng, (B, M, Hkv, D))
+        kw, vw = inputs.normal_bf16(rng, (B, W, Hkv, D)), inputs.normal_bf16(rng, (B, W, Hkv, D))
+        g.mem_load(l, binding.REGION_SLOT, dev_bf16(ks), dev_bf16(vs), first=0)
+        g.mem_load(l, binding.REGION_LOCAL, dev_bf16(kw), dev_bf16(vw), first=t0 - W)
+        kn, vn = inputs.normal_bf16(rng, (B, 1, Hkv, D)), inputs.normal_bf16(rng, (B, 1, Hkv, D))
+        h = inputs.normal_bf16(rng, (B, d))
+        Wk, Wv = inputs.normal_bf16(rng, (d, Hkv * D), d ** -0.5), inputs.normal_bf16(rng, (d, Hkv * D), d ** -0.5)
+        q = inputs.normal_bf16(rng, (B, 2, Hq, D))
+        data.append((ks, vs, kw, vw, kn, vn, h, Wk, Wv, q))
+    g.mem_set_state(t=[t0] * B, n_slots=[M] * B)
+    pos = torch.tensor([t0 + 1] * B, dtype=torch.int32, device="cuda")
+    dev = [[dev_bf16(x) for x in (kn, vn, h, Wk, Wv, q)] for (_, _, _, _, kn, vn, h, Wk, Wv, q) in data]
+    outs = [g.draft_boundary_attend(l, dev[l][0], dev[l][1], dev[l][2], dev[l][3], dev[l][4], pos, dev[l][5]) for l in range(L)]
+    torch.cuda.synchronize()
+    assert g.mem_get_state()[2] == 0
+    G, scale = Hq // Hkv, 1 / math.sqrt(D)
+    o = oracle.DraftMemory(1, B, Hq, Hkv, D, S, W, wl.slot_interval)
+    for l, (ks, vs, kw, vw, kn, vn, h, Wk, Wv, q) in enumerate(data):
+        Ko, Vo = o.materialize(0, f64(h), f64(Wk), f64(Wv), [t0 + 1] * B)
+        Kg, Vg = g.kv_view(l)
+        og, lg = outs[l]
+        for b in range(B):
+            for got, ref in ((host_bits(Kg[b, :, S + M]), Ko[b]), (host_bits(Vg[b, :, S + M]), Vo[b])):
+                assert (np.abs(f64(got) - ref) <= 2.0 ** -7 * np.abs(ref) + 1e-5).all()
+            # raw row: slots + window (oldest token left) + the new token; slot row: the same + the slot as stored
+            Kr = np.concatenate([f64(ks[b]), f64(kw[b, 1:]), f64(kn[b])]); Vr = np.concatenate([f64(vs[b]), f64(vw[b, 1:]), f64(vn[b])])
+            Ksl = np.concatenate([Kr, f64(host_bits(Kg[b, :, S + M]))[None]]); Vsl = np.concatenate([Vr, f64(host_bits(Vg[b, :, S + M]))[None]])
+            oref = np.zeros((2, Hq, D)); lref = np.zeros((2, Hq))
+            for hd in range(Hq):
+                oref[0, hd], lref[0, hd], _ = oracle.attend(f64(q[b, 0, hd]), Kr[:, hd // G], Vr[:, hd // G], scale)
+                oref[1, hd], lref[1, hd], _ = oracle.attend(f64(q[b, 1, hd]), Ksl[:, hd // G], Vsl[:, hd // G], scale)
+            assert_attention_close(og[b].cpu().numpy(), oref, lg[b].cpu().numpy(), lref, tag=f"{name} boundary layer {l}", rel_tol=2e-4)
+    g.close()
+
+
 def test_sweep_shapes_batch_and_ratio():
     """A slice of the sweep grid: batch 4 and 16, memory ratio 10 % and 50 %."""
     for wl in inputs.sweep_workloads(prefixes=(4096,), batches=(4, 16), gammas=(5,), intervals=(20, 4)):

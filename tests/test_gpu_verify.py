@@ -109,6 +109,29 @@ def test_full_size_layer_in_bench_launch_configuration(name, T):
     _case(inputs.rng_for(wl.config_id, 0, 15), wl.batch, wl.t_q_heads, wl.t_kv_heads, wl.t_head_dim, wl.prefix, T)
 
 
+def test_hints_for_a_stable_cache_and_the_next_layer_change_nothing_but_time():
+    """MASW_KV_STABLE (first tile requested ahead of the wait) and the next layer's L2 hint are scheduling hints: with
+    them a chain of layer launches gives what each launch gives alone (deterministic schedule: bit for bit), and
+    matches the oracle."""
+    rng = inputs.rng_for(5, 0, 17)
+    B, Hq, Hkv, D, P, T, L = 1, 32, 8, 128, 8192, 5, 3
+    ks = [inputs.normal_bf16(rng, (B, Hkv, P + T, D)) for _ in range(L)]
+    vs = [inputs.normal_bf16(rng, (B, Hkv, P + T, D)) for _ in range(L)]
+    qs = [inputs.normal_bf16(rng, (B, T, Hq, D)) for _ in range(L)]
+    K, V, Q = [dev_bf16(x) for x in ks], [dev_bf16(x) for x in vs], [dev_bf16(x) for x in qs]
+    kv_len = torch.tensor([P + T], dtype=torch.int32, device="cuda")
+    ws = binding.verify_workspace(K[0], kv_len, Hq, T)
+    alone = [binding.verify_attend(K[l], V[l], kv_len, Q[l], workspace=ws, deterministic=True) for l in range(L)]
+    alone = [(o.clone(), l.clone()) for o, l in alone]
+    torch.cuda.synchronize()
+    chained = [binding.verify_attend(K[l], V[l], kv_len, Q[l], workspace=ws, deterministic=True, stable_cache=True,
+                                     next_kv=(K[l + 1], V[l + 1]) if l + 1 < L else None) for l in range(L)]
+    for l in range(L):
+        assert torch.equal(chained[l][0], alone[l][0]) and torch.equal(chained[l][1], alone[l][1])
+        oref, lref = oracle.verify_attend(f64(qs[l]), f64(ks[l]), f64(vs[l]), [P + T])
+        assert_attention_close(chained[l][0].cpu().numpy(), oref, chained[l][1].cpu().numpy(), lref, tag=f"hinted chain, layer {l}")
+
+
 def test_sweep_batches():
     rng = inputs.rng_for(5, 0, 16)
     _case(rng, 4, 32, 8, 128, 4096, 2)
