@@ -127,6 +127,19 @@ __device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }
 
+// Named barrier that also ORs a predicate over its participants: every thread learns whether any of them set it.
+__device__ __forceinline__ bool named_bar_red_or(int id, int n_threads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(n_threads), "r"(static_cast<uint32_t>(pred))
+      : "memory");
+  return r != 0;
+}
+
 // Butterfly over the 32 lanes of a warp for N = 32 or 16 values per lane: on return lane L holds op over
 // all lanes of the original v[L % N] (N - 1 exchange shuffles, one more for N = 16).  `v` is destroyed.
 template <int N, bool IS_MAX>
@@ -629,8 +642,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     bool ok = true;
 
     volatile int* stop = &ctl->stop[grp];
+    constexpr float kSlack = 8.f;
+    bool refs_finite = false;   // every row of the group has a finite reference (identical in the group's threads)
     for (int i = 0;; ++i) {
       const int sb = i & 1;
+      bool exceed = false;
       if (ok) ok = mbar_wait_bounded(&ctl->s_full[sb], (i >> 1) & 1, MASW_WAIT_LIMIT(p));
       ok = __all_sync(0xffffffffu, ok);
       const int tile = ctl->tile_id[i & 15];
@@ -660,24 +676,41 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
           for (int c = 0; c < kCols; ++c) s[c] = (x <= ctl->row_hi[cg + c]) ? s[c] : kNegInf;
         }
-        // column maxima over the 128 entries: butterfly inside the warp, then across the group's four warps
-        float t[kCols];
+        // Does any score of this thread exceed its row's reference by more than the slack?  After the first few
+        // tiles the answer is almost always no for all 128 threads of the group, and then the column maxima are
+        // not needed at all: the references stay, nothing is rescaled, and the exchange below is skipped.
+        if (refs_finite) {
 #pragma unroll
-        for (int c = 0; c < kCols; ++c) t[c] = s[c];
-        ctl->colmax[i & 1][w][cg + lc] = warp_transpose_reduce<kCols, true>(t, lane);
+          for (int c4 = 0; c4 < kCols; c4 += 4) {
+            const float4 mu4 = *reinterpret_cast<const float4*>(&ctl->bcast[w][0][cg + c4]);
+            exceed |= fmaf(s[c4], p.scale_log2e, mu4.x) > kSlack || fmaf(s[c4 + 1], p.scale_log2e, mu4.y) > kSlack ||
+                      fmaf(s[c4 + 2], p.scale_log2e, mu4.z) > kSlack || fmaf(s[c4 + 3], p.scale_log2e, mu4.w) > kSlack;
+          }
+        } else {
+          exceed = true;   // some row has no finite reference yet
+        }
       } else {
         *stop = 1;
       }
-      named_bar_sync(bar_id, 128);
+      const bool move = named_bar_red_or(bar_id, 128, exceed);
       if (*stop != 0) {
         n_tiles = i;
         break;
       }
+      bool any_changed = false;
+      if (move) {
+      // column maxima over the 128 entries: butterfly inside the warp, then across the group's four warps
+      {
+        float t[kCols];
+#pragma unroll
+        for (int c = 0; c < kCols; ++c) t[c] = s[c];
+        ctl->colmax[i & 1][w][cg + lc] = warp_transpose_reduce<kCols, true>(t, lane);
+      }
+      named_bar_sync(bar_id, 128);
       // The reference each column subtracts (m_col) follows the running maximum lazily: it moves only
       // when the new maximum exceeds it by more than kSlack (in log2 units), so probabilities may reach
       // 2^kSlack instead of 1, which bf16 / fp32 hold without loss, and the O^T accumulator in tensor
       // memory has to be rescaled only on those rare moves.  o = O / l is unchanged by the choice.
-      constexpr float kSlack = 8.f;
       bool changed;
       {
         const int c = cg + lc;
@@ -690,11 +723,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         ctl->bcast[w][1][c] = changed ? fast_exp2(m_col - mu) : 1.f;
         m_col = m_new;
       }
-      const bool any_changed = __any_sync(0xffffffffu, changed);   // identical in the group's four warps
+      any_changed = __any_sync(0xffffffffu, changed);   // identical in the group's four warps
+      refs_finite = __all_sync(0xffffffffu, m_col != kNegInf);
       __syncwarp();
+      }   // if (move)
 
       // probabilities (rounded to bf16, the row sums use the rounded values)
       uint32_t pk[kCols / 2];   // packed pairs of consecutive rows
+#ifdef MASW_TRACE
+      if (p.debug_flags & 64) {   // timing experiment: no exponentials
+#pragma unroll
+        for (int c = 0; c < kCols / 2; ++c) pk[c] = 0;
+      } else
+#endif
 #pragma unroll
       for (int c4 = 0; c4 < kCols; c4 += 4) {
         const float4 mu4 = *reinterpret_cast<const float4*>(&ctl->bcast[w][0][cg + c4]);
