@@ -69,11 +69,11 @@ static int launch_attend(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendP
 
 // The draft's decode launch for up to eight query rows per KV head: one CTA per SM and launch, but a footprint
 // that lets the next layer's CTAs become resident beside this layer's (see attend_draft_kernel.cuh).
-template <int D>
+template <int D, bool PACK>
 static int launch_attend_draft(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendParams p, int B, int Hkv,
                                int tiles_upper, int splits_max, cudaStream_t st) {
   using C = DraftCfg<D>;
-  auto kern = attend_draft_kernel<D>;
+  auto kern = attend_draft_kernel<D, PACK>;
   static PerDeviceOnce once;
   {
     const int dev = current_device();
@@ -289,9 +289,15 @@ static int draft_attend_impl(masw_mem* mem, int layer, const void* k_raw, const 
     p.early = (mem->kv_clean && !(last_row_is_slot && slot.h_g == nullptr)) ? 1 : 0;
     const int te = (c.head_dim == 64) ? DraftCfg<64>::TE : DraftCfg<128>::TE;   // equals tile_entries(head_dim, 1): same tensor maps
     const int tiles_upper = (entries_upper + te - 1) / te + 4;
-    rc = (c.head_dim == 64)
-             ? launch_attend_draft<64>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, static_cast<cudaStream_t>(stream))
-             : launch_attend_draft<128>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, static_cast<cudaStream_t>(stream));
+    // at most four rows: the instance that packs both bf16 terms of the probabilities into one MMA's columns
+    const bool pack = n_q * mem->G <= 4;
+    const cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (c.head_dim == 64)
+      rc = pack ? launch_attend_draft<64, true>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st)
+                : launch_attend_draft<64, false>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st);
+    else
+      rc = pack ? launch_attend_draft<128, true>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st)
+                : launch_attend_draft<128, false>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st);
   } else {
     rc = dispatch_attend(c.head_dim, mt, tk, tv, p, c.batch, c.n_kv_heads, entries_upper, 4, mem->L.splits_max,
                          static_cast<cudaStream_t>(stream));

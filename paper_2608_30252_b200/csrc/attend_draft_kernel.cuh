@@ -13,7 +13,9 @@
 //    N: S^T[16 entries x 8 rows] = K . Q^T and O^T[16 dims x 8 rows] += V^T . P^T with mma.sync.m16n8k16, half
 //    the instructions of the rows-on-M form, and no query tile in shared memory: the Q^T fragments are loaded
 //    from global memory straight into registers.  P^T reaches its operand layout with movmatrix; it is carried
-//    as hi + lo bf16 terms, which removes the bf16 rounding of the probabilities from the result.
+//    as hi + lo bf16 terms, which removes the bf16 rounding of the probabilities from the result.  With at most
+//    four real rows (instance PACK) the two terms share one instruction: columns 4..7 of Q^T repeat rows 0..3,
+//    their threads keep the remainders, and V^T P^T accumulates head and remainder side by side.
 //
 // All eight warps consume: warp w owns tiles w, w + 8, ...  There is no producer warp: thread 0 requests the first
 // seven tiles, and the warp that has consumed tile i requests tile i + 7 into the stage it just freed.  A stage
@@ -327,7 +329,7 @@ __device__ __forceinline__ void draft_reduce_and_store(const AttendParams& p, in
   if (split == 0 && tid == 0) p.tickets[bh * (kMaxSplitsDev + 1)] = tag;
 }
 
-template <int D>
+template <int D, bool PACK>
 __global__ void __launch_bounds__(DraftCfg<D>::kThreads, 2)
 attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttendParams p) {
   using C = DraftCfg<D>;
@@ -449,6 +451,12 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   // Thread (lane / 4, lane % 4) holds row lane / 4, dims 16 ks + 2 (lane % 4) + {0, 1} and + 8.
   const int gq = lane >> 2;
   const int q2 = (lane & 3) * 2;
+  // PACK (at most four real rows): MMA columns 4..7 repeat rows 0..3, so the scores come out twice; the threads
+  // of columns 0..3 carry the bf16 head of each probability and those of columns 4..7 its bf16 remainder, and ONE
+  // V^T P^T instruction per block accumulates both terms (in columns c and c + 4, added when the warps merge)
+  const int gr = PACK ? (gq & 3) : gq;      // query row of this thread's Q^T column
+  const int qc = PACK ? (q2 & 3) : q2;      // query row of this thread's first S^T / O^T column
+  const bool lo_term = PACK && (lane & 2);  // this thread's columns carry the remainders
   uint32_t qb[D / 16][2];
   int epoch_reg = 0;   // this head's reduction epoch (every thread loads it: one broadcast transaction per warp)
   auto wait_for_predecessor_and_load_q = [&]() {
@@ -458,8 +466,8 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     MASW_STAMP(tr, 10);
     MASW_CLOCK(tr, 1);    // developer build, cycle stamps of thread 0: the wait has passed
     {
-      const bool real = gq < n_rows;
-      const int j = gq / p.G, g = gq % p.G;
+      const bool real = gr < n_rows;
+      const int j = gr / p.G, g = gr % p.G;
       const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
           p.q + ((static_cast<size_t>(b) * p.n_q + (real ? j : 0)) * p.Hq + kvh * p.G + (real ? g : 0)) * D);
 #pragma unroll
@@ -723,8 +731,8 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       mma_bf16_16816(s4, a, qb[ks][0], qb[ks][1]);
     }
     const int x = r_x0 + warp * 8 + gq;
-    const bool v0 = warp < TE / 8 && x >= ctl->row_lo[r_seg * 8 + q2] && x <= ctl->row_hi[r_seg * 8 + q2];
-    const bool v1 = warp < TE / 8 && x >= ctl->row_lo[r_seg * 8 + q2 + 1] && x <= ctl->row_hi[r_seg * 8 + q2 + 1];
+    const bool v0 = warp < TE / 8 && x >= ctl->row_lo[r_seg * 8 + qc] && x <= ctl->row_hi[r_seg * 8 + qc];
+    const bool v1 = warp < TE / 8 && x >= ctl->row_lo[r_seg * 8 + qc + 1] && x <= ctl->row_hi[r_seg * 8 + qc + 1];
     const float s0 = v0 ? s4[0] * p.scale_log2e : kNegInf;
     const float s1 = v1 ? s4[1] * p.scale_log2e : kNegInf;
     float mx0 = s0, mx1 = s1;
@@ -738,12 +746,21 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     l_run[0] = p0; l_run[1] = p1;
     const uint32_t ha = pack_bf16x2(p0, p1);
     const float r0 = __uint_as_float(ha << 16), r1 = __uint_as_float(ha & 0xffff0000u);
-    const uint32_t bh = movmatrix_trans(ha), bl = movmatrix_trans(pack_bf16x2(p0 - r0, p1 - r1));
+    if constexpr (PACK) {
+      const uint32_t bx = movmatrix_trans(lo_term ? pack_bf16x2(p0 - r0, p1 - r1) : ha);
 #pragma unroll
-    for (int md = 0; md < D / 16; ++md) {
-      const uint32_t a[4] = {vf[md][0], vf[md][1], 0u, 0u};
-      mma_bf16_16816(acc[md], a, bh, 0u);
-      mma_bf16_16816(acc[md], a, bl, 0u);
+      for (int md = 0; md < D / 16; ++md) {
+        const uint32_t a[4] = {vf[md][0], vf[md][1], 0u, 0u};
+        mma_bf16_16816(acc[md], a, bx, 0u);
+      }
+    } else {
+      const uint32_t bh = movmatrix_trans(ha), bl = movmatrix_trans(pack_bf16x2(p0 - r0, p1 - r1));
+#pragma unroll
+      for (int md = 0; md < D / 16; ++md) {
+        const uint32_t a[4] = {vf[md][0], vf[md][1], 0u, 0u};
+        mma_bf16_16816(acc[md], a, bh, 0u);
+        mma_bf16_16816(acc[md], a, bl, 0u);
+      }
     }
   }
 
@@ -765,8 +782,8 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       for (int u = 0; u < kPre; ++u) pre[u] = n_pre[u];
       if (seg != seg_bounds) {
         seg_bounds = seg;
-        lo0 = ctl->row_lo[seg * 8 + q2]; hi0 = ctl->row_hi[seg * 8 + q2];
-        lo1 = ctl->row_lo[seg * 8 + q2 + 1]; hi1 = ctl->row_hi[seg * 8 + q2 + 1];
+        lo0 = ctl->row_lo[seg * 8 + qc]; hi0 = ctl->row_hi[seg * 8 + qc];
+        lo1 = ctl->row_lo[seg * 8 + qc + 1]; hi1 = ctl->row_hi[seg * 8 + qc + 1];
       }
       const int stage = i % NS;
       const uint32_t parity = (i / NS) & 1;
@@ -892,7 +909,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       // ---- P^T as the B operand of O^T += V^T P^T: the S^T fragment holds (entry = lane / 4, rows q2, q2 + 1);
       //      the operand wants (entries q2, q2 + 1; row = lane / 4): one 8 x 8 transpose per half block.
       //      p = p_hi + p_lo (two bf16 terms); the row sums use the unrounded values.
-      uint32_t ph[TE / 16][2], pl[TE / 16][2];
+      uint32_t ph[TE / 16][2], pl[PACK ? 1 : TE / 16][2];   // PACK: ph holds head | remainder columns, pl is unused
 #pragma unroll
       for (int mt = 0; mt < TE / 16; ++mt) {
         const float p0 = fast_exp2(st[mt][0] - mu0), p1 = fast_exp2(st[mt][1] - mu1);
@@ -902,10 +919,15 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t ha = pack_bf16x2(p0, p1), hb = pack_bf16x2(p2, p3);
         const float r0 = __uint_as_float(ha << 16), r1 = __uint_as_float(ha & 0xffff0000u);
         const float r2 = __uint_as_float(hb << 16), r3 = __uint_as_float(hb & 0xffff0000u);
-        ph[mt][0] = movmatrix_trans(ha);
-        ph[mt][1] = movmatrix_trans(hb);
-        pl[mt][0] = movmatrix_trans(pack_bf16x2(p0 - r0, p1 - r1));
-        pl[mt][1] = movmatrix_trans(pack_bf16x2(p2 - r2, p3 - r3));
+        if constexpr (PACK) {
+          ph[mt][0] = movmatrix_trans(lo_term ? pack_bf16x2(p0 - r0, p1 - r1) : ha);
+          ph[mt][1] = movmatrix_trans(lo_term ? pack_bf16x2(p2 - r2, p3 - r3) : hb);
+        } else {
+          ph[mt][0] = movmatrix_trans(ha);
+          ph[mt][1] = movmatrix_trans(hb);
+          pl[mt][0] = movmatrix_trans(pack_bf16x2(p0 - r0, p1 - r1));
+          pl[mt][1] = movmatrix_trans(pack_bf16x2(p2 - r2, p3 - r3));
+        }
       }
 
       MASW_CLOCK(tr, 17);   // ... probabilities in operand layout
@@ -925,7 +947,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             uint32_t a[4];
             ldmatrix_x4_trans(a[0], a[1], a[2], a[3], vs_base + (cg >> 3) * C::kSubBytes + e * 128 + (((cg & 7) ^ (e & 7)) << 4));
             mma_bf16_16816(acc[md], a, ph[mt][0], ph[mt][1]);
-            mma_bf16_16816(acc[md], a, pl[mt][0], pl[mt][1]);
+            if constexpr (!PACK) mma_bf16_16816(acc[md], a, pl[mt][0], pl[mt][1]);
           }
         }
       }
@@ -1018,7 +1040,11 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       for (int e = 0; e < NW; ++e) {
         const float me = mml[(e * C::kRows + r) * 2];
         const float w = (me == kNegInf) ? 0.f : fast_exp2(me - m);
-        const float4 v = *reinterpret_cast<const float4*>(mo + (e * C::kRows + r) * kMS + d4);
+        float4 v = *reinterpret_cast<const float4*>(mo + (e * C::kRows + r) * kMS + d4);
+        if constexpr (PACK) {   // columns r + 4 accumulated the remainder terms of row r
+          const float4 v2 = *reinterpret_cast<const float4*>(mo + (e * C::kRows + r + 4) * kMS + d4);
+          v.x += v2.x; v.y += v2.y; v.z += v2.z; v.w += v2.w;
+        }
         o4.x += w * v.x; o4.y += w * v.y; o4.z += w * v.z; o4.w += w * v.w;
         l += w * mml[(e * C::kRows + r) * 2 + 1];
       }
