@@ -1051,7 +1051,7 @@ def run_timeline(args, wl):
                    **{name: f"{np.median(cols[:, c]):.2f} ({cols[:, c].min():.2f}-{cols[:, c].max():.2f})"
                       for c, name in enumerate(["cta_start", "wait_passed", "end"])}}
             # thread 0's cycle stamps, as microseconds after its wait passed
-            names = [("projection_loads_issued", 23), ("projection_summed", 24), ("q_arrived", 2), ("warp0_tile_landed", 3), ("warp0_scores", 16), ("warp0_probabilities", 17), ("warp0_pv", 18),
+            names = [("reached_the_wait", 14), ("projection_loads_issued", 23), ("projection_summed", 24), ("q_arrived", 2), ("warp0_tile_landed", 3), ("warp0_scores", 16), ("warp0_probabilities", 17), ("warp0_pv", 18),
                      ("warp0_tile_done", 19), ("tiles_consumed", 8), ("partials_in_smem", 20), ("published", 9),
                      ("reduction_starts", 26), ("slot_records_first_answer", 29), ("slot_records_summed", 25), ("slot_final", 27), ("slot_phase_over", 28),
                      ("first_item_complete", 11), ("all_items_complete", 12), ("combined", 21), ("outputs_stored", 22), ("end", 13)]

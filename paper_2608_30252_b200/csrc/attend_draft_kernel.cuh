@@ -461,6 +461,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   int epoch_reg = 0;   // this head's reduction epoch (every thread loads it: one broadcast transaction per warp)
   auto wait_for_predecessor_and_load_q = [&]() {
     // a launch that was allowed to start early waits here for its predecessor, and lets its own successor start
+    MASW_CLOCK(tr, 14);   // developer build: thread 0 reaches the wait (its work ahead of the predecessor is done)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     MASW_STAMP(tr, 10);

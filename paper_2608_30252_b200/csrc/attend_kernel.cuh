@@ -122,26 +122,28 @@ __device__ __forceinline__ int build_segments(const AttendParams& p, int b, Segm
 // Every value a CTA publishes for the other splits travels as a 64-bit record: the 32-bit payload and the
 // 32-bit epoch tag of the launch that wrote it.  A 64-bit access is single-copy atomic, so a reader that
 // sees this launch's tag also sees the payload: no fence, flag or atomic is needed between writer and
-// reader, and a reader simply reloads a record until its tag is the expected one (bounded).
+// reader, and a reader simply reloads a record until its tag is the expected one (bounded).  Both sides use
+// relaxed operations at gpu scope: a cache operator (.cg) is only a hint, and a weak load repeated in a tight
+// loop may be answered by the SM's own cache for as long as the loop runs.
 __device__ __forceinline__ unsigned long long rec_make(float v, int tag) {
   return static_cast<unsigned long long>(__float_as_uint(v)) | (static_cast<unsigned long long>(static_cast<unsigned>(tag)) << 32);
 }
 __device__ __forceinline__ void rec_store1(unsigned long long* dst, float a, int tag) {
-  asm volatile("st.global.cg.u64 [%0], %1;" ::"l"(dst), "l"(rec_make(a, tag)) : "memory");
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(dst), "l"(rec_make(a, tag)) : "memory");
 }
 __device__ __forceinline__ void rec_store2(unsigned long long* dst, float a, float b, int tag) {   // 16-byte aligned
-  asm volatile("st.global.cg.v2.u64 [%0], {%1, %2};" ::"l"(dst), "l"(rec_make(a, tag)), "l"(rec_make(b, tag)) : "memory");
+  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(dst), "l"(rec_make(a, tag)), "l"(rec_make(b, tag)) : "memory");
 }
 struct Rec1 { float a; bool ok; };
 struct Rec2 { float a, b; bool ok; };
 __device__ __forceinline__ Rec1 rec_load1(const unsigned long long* src, int tag) {
   unsigned long long r;
-  asm volatile("ld.global.cg.u64 %0, [%1];" : "=l"(r) : "l"(src) : "memory");
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(r) : "l"(src) : "memory");
   return Rec1{__uint_as_float(static_cast<unsigned>(r)), static_cast<int>(r >> 32) == tag};
 }
 __device__ __forceinline__ Rec2 rec_load2(const unsigned long long* src, int tag) {   // 16-byte aligned
   unsigned long long r0, r1;
-  asm volatile("ld.global.cg.v2.u64 {%0, %1}, [%2];" : "=l"(r0), "=l"(r1) : "l"(src) : "memory");
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(r0), "=l"(r1) : "l"(src) : "memory");
   return Rec2{__uint_as_float(static_cast<unsigned>(r0)), __uint_as_float(static_cast<unsigned>(r1)),
               static_cast<int>(r0 >> 32) == tag && static_cast<int>(r1 >> 32) == tag};
 }
