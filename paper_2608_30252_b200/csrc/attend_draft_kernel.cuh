@@ -383,8 +383,10 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       }
       plan[32 + nseg] = acc;
       plan[0] = nseg;
-      plan[1] = static_cast<int>((static_cast<long long>(acc) * split) / p.splits);
-      plan[2] = static_cast<int>((static_cast<long long>(acc) * (split + 1)) / p.splits);
+      // split s takes tiles [ceil(acc s / splits), ceil(acc (s + 1) / splits)): where the tiles do not divide evenly
+      // the LAST split, which also patches the pending raw rows into its last tile, is among the short ones
+      plan[1] = static_cast<int>((static_cast<long long>(acc) * split + p.splits - 1) / p.splits);
+      plan[2] = static_cast<int>((static_cast<long long>(acc) * (split + 1) + p.splits - 1) / p.splits);
       plan[3] = 0;
       plan[7] = t_b;
     }
@@ -393,8 +395,8 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       int acc = 0;
       for (int s = 0; s < nseg; ++s) { first[s] = acc; acc += (seg[s].len + TE - 1) / TE; }
       first[nseg] = acc;
-      const int tb = static_cast<int>((static_cast<long long>(acc) * split) / p.splits);
-      const int te = static_cast<int>((static_cast<long long>(acc) * (split + 1)) / p.splits);
+      const int tb = static_cast<int>((static_cast<long long>(acc) * split + p.splits - 1) / p.splits);
+      const int te = static_cast<int>((static_cast<long long>(acc) * (split + 1) + p.splits - 1) / p.splits);
       const uint64_t policy = l2_policy_evict_first();
       const int n0 = min(te - tb, NS);
       int sg = 0;
