@@ -511,6 +511,31 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   // Without p.early everything follows the wait.  With it, the plan and the first ring of copies come first and
   // only q, the pending raw rows and the epoch are read behind the wait: the tiles are in shared memory by then.
   if (!p.early) {
+    // The launch in front may still be writing the counters (a counter update, a rollback) or the arena, so
+    // nothing is READ for use ahead of the wait.  But this CTA's tiles can be asked into L2 from a guess: the
+    // counters as they stand now (one step old at worst) name almost the same entries, a prefetch returns no
+    // data, and a wrong guess costs nothing but the hint.  The real plan follows behind the wait.
+    if (is_producer) {
+      Segment seg[kMaxSeg];
+      int t_g, m_g;
+      const int nseg_g = build_segments<true>(p, b, seg, t_g, m_g);
+      int first[kMaxSeg + 1];
+      int acc = 0;
+      for (int s = 0; s < nseg_g; ++s) { first[s] = acc; acc += (seg[s].len + TE - 1) / TE; }
+      first[nseg_g] = acc;
+      const int tb = static_cast<int>((static_cast<long long>(acc) * split + p.splits - 1) / p.splits);
+      const int te = static_cast<int>((static_cast<long long>(acc) * (split + 1) + p.splits - 1) / p.splits);
+      int sg = 0;
+      for (int it = tb; it < min(te, tb + NS + 1); ++it) {
+        while (sg + 1 < nseg_g && it >= first[sg + 1]) ++sg;
+        const int row0 = seg[sg].phys + (it - first[sg]) * TE;
+#pragma unroll
+        for (int sub = 0; sub < C::kSub; ++sub) {
+          tma_prefetch_4d(&tmK, sub * 64, row0, kvh, b);
+          tma_prefetch_4d(&tmV, sub * 64, row0, kvh, b);
+        }
+      }
+    }
     wait_for_predecessor_and_load_q();
     if (proj_on) proj_load_weights(pk0 + prl);
   }

@@ -85,18 +85,28 @@ struct Segment {
 // Enumerates the contiguous runs of physical entries that some row of this sequence may read.
 // Draft (Eq. 3): sink [0,S) | committed (+ pending) slots | the ring pieces holding the union of the
 // rows' local windows.  Verify: the cache prefix [0, kv_len).
+// HINT: the counters are read with relaxed gpu-scope loads, which leave no line in the SM's own cache: the
+// caller runs ahead of a launch that may still be writing them and wants only a guess (for L2 prefetches); it
+// reads them again, the ordinary way, once its predecessor has completed.
+__device__ __forceinline__ int ld_counter(const int* ptr, bool hint) {
+  if (!hint) return *ptr;
+  int v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+template <bool HINT = false>
 __device__ __forceinline__ int build_segments(const AttendParams& p, int b, Segment (&seg)[kMaxSeg], int& t_out,
                                               int& m_out) {
   int n = 0;
   if (p.kv_len != nullptr) {
-    int len = min(max(p.kv_len[b], 0), p.capacity);
+    int len = min(max(ld_counter(p.kv_len + b, HINT), 0), p.capacity);
     t_out = len;
     m_out = 0;
     if (len > 0) seg[n++] = Segment{0, len, 0, 2};
     return n;
   }
-  const int t = p.t[b];
-  const int M = p.n_slots[b];
+  const int t = max(ld_counter(p.t + b, HINT), 0);
+  const int M = min(max(ld_counter(p.n_slots + b, HINT), 0), p.max_slots);
   t_out = t;
   m_out = M;
   const int n_raw = p.n_q - p.last_row_is_slot;

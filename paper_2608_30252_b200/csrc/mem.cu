@@ -159,6 +159,11 @@ slot_project_kernel(__nv_bfloat16* K, __nv_bfloat16* V, const __nv_bfloat16* h_g
 
 __global__ void advance_kernel(int* t, int* n_slots, int* status, const uint8_t* active, int B, int n_tokens,
                                int add_slot, int max_slots) {
+  // Launched with programmatic stream serialisation: the next launch (an attention layer, which reads the
+  // counters only behind its own wait) may be set up at once, and the counters are written only when the
+  // launch in front of this one, which still reads them, has completed.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   t[b] += n_tokens;
@@ -169,6 +174,8 @@ __global__ void advance_kernel(int* t, int* n_slots, int* status, const uint8_t*
 }
 
 __global__ void rollback_kernel(int* t, int* n_slots, const int* t_keep, const int* slots_keep, int B) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // as in advance_kernel
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   t[b] = max(0, min(t[b], t_keep[b]));
@@ -389,10 +396,20 @@ extern "C" int mem_advance(masw_mem* mem, int n_tokens, int add_slot, const uint
     mem->slots_upper += 1;
   }
   const int B = mem->cfg.batch;
-  advance_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
-      mem->d_t, mem->d_slots, mem->d_status, active, B, n_tokens, add_slot ? 1 : 0, mem->cfg.max_slots);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((B + 127) / 128, 1, 1);
+    cfg.blockDim = dim3(128, 1, 1);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, advance_kernel, mem->d_t, mem->d_slots, mem->d_status, active, B, n_tokens,
+                                     add_slot ? 1 : 0, mem->cfg.max_slots));
+  }
   count_launch();
-  MASW_CUDA_TRY(cudaGetLastError());
   return MASW_OK;
 }
 
@@ -402,8 +419,18 @@ extern "C" int mem_rollback(masw_mem* mem, const int32_t* t_keep, const int32_t*
   mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   if (slots_keep_max >= 0) mem->slots_upper = std::min(mem->slots_upper, slots_keep_max);
   const int B = mem->cfg.batch;
-  rollback_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(mem->d_t, mem->d_slots, t_keep, slots_keep, B);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((B + 127) / 128, 1, 1);
+    cfg.blockDim = dim3(128, 1, 1);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, rollback_kernel, mem->d_t, mem->d_slots, t_keep, slots_keep, B));
+  }
   count_launch();
-  MASW_CUDA_TRY(cudaGetLastError());
   return MASW_OK;
 }
