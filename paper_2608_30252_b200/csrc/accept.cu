@@ -159,15 +159,16 @@ accept_reject_kernel(const unsigned short* tl, const unsigned short* dl, const i
     if (vec) {
       const uint4* row4 = reinterpret_cast<const uint4*>(row);
       const int n4 = V / 8;
-      for (int j0 = tid; j0 < n4; j0 += kAcceptThreads * 4) {
-        uint4 w[4];
+      constexpr int kInFlight = 8;   // 16-byte loads per thread and round trip (a 128K-entry row takes four trips)
+      for (int j0 = tid; j0 < n4; j0 += kAcceptThreads * kInFlight) {
+        uint4 w[kInFlight];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kInFlight; ++u) {
           const int j4 = j0 + u * kAcceptThreads;
           w[u] = j4 < n4 ? __ldg(row4 + j4) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // -inf pads
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kInFlight; ++u) {
           const int j4 = j0 + u * kAcceptThreads;
           if (j4 >= n4) continue;
           const unsigned int word[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
