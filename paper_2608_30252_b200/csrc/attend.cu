@@ -3,6 +3,8 @@
 #include <mutex>
 #include <vector>
 
+#include <type_traits>
+
 #include "attend_draft_kernel.cuh"
 #include "attend_kernel.cuh"
 #include "attend_tc_kernel.cuh"
@@ -69,11 +71,11 @@ static int launch_attend(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendP
 
 // The draft's decode launch for up to eight query rows per KV head: one CTA per SM and launch, but a footprint
 // that lets the next layer's CTAs become resident beside this layer's (see attend_draft_kernel.cuh).
-template <int D, bool PACK>
+template <int D, bool PACK, bool SLOT>
 static int launch_attend_draft(const CUtensorMap& tmK, const CUtensorMap& tmV, AttendParams p, int B, int Hkv,
                                int tiles_upper, int splits_max, cudaStream_t st) {
   using C = DraftCfg<D>;
-  auto kern = attend_draft_kernel<D, PACK>;
+  auto kern = attend_draft_kernel<D, PACK, SLOT>;
   static PerDeviceOnce once;
   {
     const int dev = current_device();
@@ -292,12 +294,21 @@ static int draft_attend_impl(masw_mem* mem, int layer, const void* k_raw, const 
     // at most four rows: the instance that packs both bf16 terms of the probabilities into one MMA's columns
     const bool pack = n_q * mem->G <= 4;
     const cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c.head_dim == 64)
-      rc = pack ? launch_attend_draft<64, true>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st)
-                : launch_attend_draft<64, false>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st);
-    else
-      rc = pack ? launch_attend_draft<128, true>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st)
-                : launch_attend_draft<128, false>(tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st);
+    const bool fused_slot = p.h_g != nullptr;   // the instance with the boundary step's slot materialisation
+    auto go = [&](auto d, auto pk, auto sl) {
+      return launch_attend_draft<decltype(d)::value, decltype(pk)::value, decltype(sl)::value>(
+          tk, tv, p, c.batch, c.n_kv_heads, tiles_upper, mem->L.splits_max, st);
+    };
+    using std::integral_constant;
+    using T = std::true_type;
+    using F = std::false_type;
+    if (c.head_dim == 64) {
+      using Dn = integral_constant<int, 64>;
+      rc = pack ? (fused_slot ? go(Dn{}, T{}, T{}) : go(Dn{}, T{}, F{})) : (fused_slot ? go(Dn{}, F{}, T{}) : go(Dn{}, F{}, F{}));
+    } else {
+      using Dn = integral_constant<int, 128>;
+      rc = pack ? (fused_slot ? go(Dn{}, T{}, T{}) : go(Dn{}, T{}, F{})) : (fused_slot ? go(Dn{}, F{}, T{}) : go(Dn{}, F{}, F{}));
+    }
   } else {
     rc = dispatch_attend(c.head_dim, mt, tk, tv, p, c.batch, c.n_kv_heads, entries_upper, 4, mem->L.splits_max,
                          static_cast<cudaStream_t>(stream));

@@ -16,6 +16,8 @@
 //    as hi + lo bf16 terms, which removes the bf16 rounding of the probabilities from the result.  With at most
 //    four real rows (instance PACK) the two terms share one instruction: columns 4..7 of Q^T repeat rows 0..3,
 //    their threads keep the remainders, and V^T P^T accumulates head and remainder side by side.
+//  Instance SLOT carries the fused slot materialisation of the boundary step (h_g given); the plain decode launch
+//  is compiled without it, so that its registers and its schedule do not pay for code it never runs.
 //
 // All eight warps consume: warp w owns tiles w, w + 8, ...  There is no producer warp: thread 0 requests the first
 // seven tiles, and the warp that has consumed tile i requests tile i + 7 into the stage it just freed.  A stage
@@ -88,7 +90,7 @@ __device__ __forceinline__ void st_release_shared(int* p, int v) {
 // split order, rotate the key, round both to bf16 as stored and take the slot rows' scores against it while the
 // other splits are still publishing; behind the rendezvous only the final combine is left.
 // Must be called by all 256 threads; `scratch` is shared memory of at least 9 KB + 24 D bytes.
-template <int D>
+template <int D, bool SLOT>
 __device__ __forceinline__ void draft_reduce_and_store(const AttendParams& p, int b, int kvh, int split, int n_rows, int epoch,
                                                        float* scratch, int tid, const float* rope_cs, long long* tr) {
   constexpr float kNegInf = -INFINITY;
@@ -116,7 +118,7 @@ __device__ __forceinline__ void draft_reduce_and_store(const AttendParams& p, in
   // attention partials (the splits published their sums of K_g | V_g at the start of the launch, so these
   // records have long arrived; the loads ride along with the wait for the other splits' partials)
   const int first_slot_item = (n_rows - p.G) * (D / 4);
-  const bool slot_term = p.h_g != nullptr && (p.active == nullptr || p.active[b] != 0) &&
+  const bool slot_term = SLOT && p.h_g != nullptr && (p.active == nullptr || p.active[b] != 0) &&
                          (split == 0 || i_begin + my_items > first_slot_item);
   constexpr int kColGroups = NT / D;                        // thread (columns 2 c, 2 c + 1 of K | V, group): splits group, group + groups, ...
   constexpr int kBatch = (D == 64) ? 5 : 10;                // 16-byte record pairs in flight per thread: up to 20 splits in one round trip
@@ -329,7 +331,7 @@ __device__ __forceinline__ void draft_reduce_and_store(const AttendParams& p, in
   if (split == 0 && tid == 0) p.tickets[bh * (kMaxSplitsDev + 1)] = tag;
 }
 
-template <int D, bool PACK>
+template <int D, bool PACK, bool SLOT>
 __global__ void __launch_bounds__(DraftCfg<D>::kThreads, 2)
 attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttendParams p) {
   using C = DraftCfg<D>;
@@ -491,7 +493,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   constexpr int kProjChunks = kProjColsPerWarp / 8;   // 16-byte chunks of a row this warp reads: 2 or 4
   constexpr int kProjRowLanes = 32 / kProjChunks;
   constexpr int kProjInFlight = 8;                    // weight rows per lane and round trip
-  const bool proj_on = p.h_g != nullptr && (p.active == nullptr || p.active[b] != 0);
+  const bool proj_on = SLOT && p.h_g != nullptr && (p.active == nullptr || p.active[b] != 0);
   const int prl = lane / kProjChunks;
   const int pcol = warp * kProjColsPerWarp + (lane % kProjChunks) * 8;   // first of this lane's eight columns in K | V
   const int pk0 = static_cast<int>((static_cast<long long>(p.d_model) * split) / p.splits);
@@ -540,7 +542,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (proj_on) proj_load_weights(pk0 + prl);
   }
   plan_and_issue();
-  if (warp == NW - 1 && p.h_g != nullptr) {
+  if (SLOT && warp == NW - 1 && p.h_g != nullptr) {
 #pragma unroll
     for (int u = 0; u < kRopePerLane; ++u) {
       const int i = lane + 32 * u;
@@ -1092,7 +1094,7 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 #else
   long long* tr = nullptr;
 #endif
-  draft_reduce_and_store<D>(p, b, kvh, split, n_rows, plan[6], reinterpret_cast<float*>(pipe + C::kReduceOff), tid, rope_cs, tr);
+  draft_reduce_and_store<D, SLOT>(p, b, kvh, split, n_rows, plan[6], reinterpret_cast<float*>(pipe + C::kReduceOff), tid, rope_cs, tr);
   MASW_CLOCK(tr, 13);
   MASW_STAMP(tr, 4);
 }
