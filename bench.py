@@ -126,6 +126,7 @@ class StepRunner:
         self.host_in = torch.empty(self.in_bytes, dtype=torch.uint8).pin_memory()
         self._fill_host_inputs()
         self.dev_in.copy_(self.host_in)
+        self.e2e_graph = None   # captured by the first end-to-end step
 
         # ---- outputs
         self.d_o1 = torch.empty((wl.d_layers, B, 1, wl.d_q_heads, wl.d_head_dim), dtype=torch.float32, device=device)
@@ -222,16 +223,39 @@ class StepRunner:
         if events is not None:
             events[3].record()
 
-    def step_e2e(self):
-        """One iteration through host buffers: pinned H2D of the step's inputs, the three phases, D2H of
-        the decision (accepted length and tokens), then a stream synchronisation."""
+    def capture_e2e(self):
+        """The end-to-end iteration as ONE CUDA graph: the pinned host -> device copies of the step's inputs (on a
+        forked copy stream, one copy per phase in the order the phases read them; a phase depends on its own copy
+        only, so the verifier's queries and the logits cross the bus while the draft steps run), the three phases,
+        and the device -> host copy of the decision."""
         torch = self.torch
-        self.dev_in.copy_(self.host_in, non_blocking=True)
-        for g in self.graphs:
-            g.replay()
-        self.host_out[:, 0].copy_(self.n_acc, non_blocking=True)
-        self.host_out[:, 1:].copy_(self.out_tok, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        copy_stream = torch.cuda.Stream(device=self.dev)
+        events = [torch.cuda.Event() for _ in range(3)]
+        cuts = [0, self.fields["vq"][0], self.fields["tl"][0], self.in_bytes]   # draft | verify | tail inputs
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            main = torch.cuda.current_stream()
+            copy_stream.wait_stream(main)
+            with torch.cuda.stream(copy_stream):
+                for a, b, ev in zip(cuts[:-1], cuts[1:], events):
+                    self.dev_in[a:b].copy_(self.host_in[a:b], non_blocking=True)
+                    ev.record(copy_stream)
+            for phase, ev in zip((self.draft_phase, self.verify_phase, self.tail_phase), events):
+                main.wait_event(ev)
+                phase()
+            self.host_out[:, 0].copy_(self.n_acc, non_blocking=True)
+            self.host_out[:, 1:].copy_(self.out_tok, non_blocking=True)
+            main.wait_stream(copy_stream)
+        self.e2e_graph = g
+        torch.cuda.synchronize()
+
+    def step_e2e(self):
+        """One iteration through host buffers (one graph launch: copies in, the three phases, the decision out),
+        then a stream synchronisation: the host holds the step's result when this returns."""
+        if self.e2e_graph is None:
+            self.capture_e2e()
+        self.e2e_graph.replay()
+        self.torch.cuda.current_stream().synchronize()
 
 
 def draft_comparators(wl, device, reps=20):
@@ -648,7 +672,10 @@ def run_gpu(args, wl):
                        "target": f"{wl.t_layers}L {wl.t_q_heads}q/{wl.t_kv_heads}kv d{wl.t_head_dim}, full KV",
                        "step": f"{g} draft steps (slot materialisation on one of them) + verify of {g} rows + "
                                f"greedy accept/reject (V={wl.vocab}) + rollback; replicas only at n_gpus > 1",
-                       "l2": "inputs larger than L2 (step reads %.2f GB of KV)" % ((draft_bytes_step * g + verify_bytes) / 1e9)},
+                       "l2": "inputs larger than L2 (step reads %.2f GB of KV)" % ((draft_bytes_step * g + verify_bytes) / 1e9),
+                       "e2e_step": "one CUDA graph per step: pinned host -> device copies on a forked copy stream, one per phase "
+                                   "(a phase depends on its own copy only), the three phases, the decision device -> host; "
+                                   "the host synchronises after every step"},
             "phases": {"draft_us_per_draft_step": draft_us, "draft_us_per_layer": draft_us / wl.d_layers,
                        "draft_kv_gbs": d_gbs, "draft_frac_of_8tbs": d_gbs / 8000.0, "draft_frac_of_measured": d_gbs / peak,
                        "draft_kv_bytes_per_step": draft_bytes_step,
