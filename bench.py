@@ -135,9 +135,11 @@ class StepRunner:
         self.d_lse2 = torch.empty((wl.d_layers, B, 2, wl.d_q_heads), dtype=torch.float32, device=device)
         self.v_o = torch.empty((wl.t_layers, B, g, wl.t_q_heads, wl.t_head_dim), dtype=torch.float32, device=device)
         self.v_lse = torch.empty((wl.t_layers, B, g, wl.t_q_heads), dtype=torch.float32, device=device)
-        self.n_acc = torch.empty((B,), dtype=torch.int32, device=device)
-        self.out_tok = torch.empty((B, g + 1), dtype=torch.int32, device=device)
-        self.host_out = torch.empty((B, g + 2), dtype=torch.int32).pin_memory()
+        # the decision of a step: accepted lengths [B], then emitted tokens [B][g + 1], in one buffer (one copy back)
+        self.out_dev = torch.empty((B * (g + 2),), dtype=torch.int32, device=device)
+        self.n_acc = self.out_dev[:B]
+        self.out_tok = self.out_dev[B:].view(B, g + 1)
+        self.host_out = torch.empty((B * (g + 2),), dtype=torch.int32).pin_memory()
         self.out_bytes = self.host_out.numel() * 4
         self.v_ws = binding.verify_workspace(self.tK[0], self.kv_len, wl.t_q_heads, g)
         self.a_ws = binding.accept_workspace(B, g, wl.vocab, device)
@@ -169,9 +171,9 @@ class StepRunner:
             self.host_in[off:off + n * t.element_size()].copy_(t.view(torch.uint8).reshape(-1))
 
     # ---- the three phases of one speculative iteration, as C-ABI calls on the current stream
-    def draft_phase(self):
+    def draft_phase(self, steps=None):
         wl, mem = self.wl, self.mem
-        for j in range(wl.gamma):
+        for j in (range(wl.gamma) if steps is None else steps):
             fire = (j == self.slot_step)
             q, k, v = self.view(f"dq{j}"), self.view(f"dk{j}"), self.view(f"dv{j}")
             for l in range(wl.d_layers):
@@ -241,25 +243,31 @@ class StepRunner:
     def capture_e2e(self):
         """The end-to-end iteration as ONE CUDA graph: the pinned host -> device copies of the step's inputs (on a
         forked copy stream, one copy per phase in the order the phases read them; a phase depends on its own copy
-        only, so the verifier's queries and the logits cross the bus while the draft steps run), the three phases,
+        only, so all but the first draft step's inputs cross the bus while earlier stages run), the three phases,
         and the device -> host copy of the decision."""
         torch = self.torch
         copy_stream = torch.cuda.Stream(device=self.dev)
-        events = [torch.cuda.Event() for _ in range(3)]
-        cuts = [0, self.fields["vq"][0], self.fields["tl"][0], self.in_bytes]   # draft | verify | tail inputs
+        # copies in the order they are needed: the first draft step's inputs, the other draft steps' (and h_g), the
+        # verifier's queries, the logits and proposals
+        first = self.fields["dq1"][0] if (self.wl.gamma > 1 and self.slot_step > 0) else self.fields["vq"][0]
+        cuts = [0, first, self.fields["vq"][0], self.fields["tl"][0], self.in_bytes]
+        events = [torch.cuda.Event() for _ in range(4)]
+        rest = range(1, self.wl.gamma) if first != cuts[2] else range(0)
+        stages = [lambda: self.draft_phase(range(0, 1) if first != cuts[2] else None),
+                  lambda: self.draft_phase(rest), self.verify_phase, self.tail_phase]
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             main = torch.cuda.current_stream()
             copy_stream.wait_stream(main)
             with torch.cuda.stream(copy_stream):
                 for a, b, ev in zip(cuts[:-1], cuts[1:], events):
-                    self.dev_in[a:b].copy_(self.host_in[a:b], non_blocking=True)
+                    if b > a:
+                        self.dev_in[a:b].copy_(self.host_in[a:b], non_blocking=True)
                     ev.record(copy_stream)
-            for phase, ev in zip((self.draft_phase, self.verify_phase, self.tail_phase), events):
+            for stage, ev in zip(stages, events):
                 main.wait_event(ev)
-                phase()
-            self.host_out[:, 0].copy_(self.n_acc, non_blocking=True)
-            self.host_out[:, 1:].copy_(self.out_tok, non_blocking=True)
+                stage()
+            self.host_out.copy_(self.out_dev, non_blocking=True)
             main.wait_stream(copy_stream)
         self.e2e_graph = g
         torch.cuda.synchronize()
@@ -665,6 +673,9 @@ def run_gpu(args, wl):
     barrier()
     e2e_ms = es.elapsed_time(ee)
     e2e_wall_ms = (time.perf_counter() - tic) * 1e3
+    # the decision the host received is the one on the device, and an accepted length is in range
+    assert torch.equal(runner.host_out, runner.out_dev.cpu()), "end-to-end step: host copy of the decision differs"
+    assert 0 <= int(runner.host_out[: wl.batch].min()) and int(runner.host_out[: wl.batch].max()) <= wl.gamma
     _, _, status = runner.mem.mem_get_state()
 
     total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], device=dev)
@@ -705,9 +716,10 @@ def run_gpu(args, wl):
                        "step": f"{g} draft steps (slot materialisation on one of them) + verify of {g} rows + "
                                f"greedy accept/reject (V={wl.vocab}) + rollback; replicas only at n_gpus > 1",
                        "l2": "inputs larger than L2 (step reads %.2f GB of KV)" % ((draft_bytes_step * g + verify_bytes) / 1e9),
-                       "e2e_step": "one CUDA graph per step: pinned host -> device copies on a forked copy stream, one per phase "
-                                   "(a phase depends on its own copy only), the three phases, the decision device -> host; "
-                                   "the host synchronises after every step"},
+                       "e2e_step": "one CUDA graph per step: pinned host -> device copies on a forked copy stream in the order "
+                                   "they are needed (first draft step's inputs, the other draft steps', the verifier's "
+                                   "queries, logits and proposals; a stage depends on its own copy only), the three "
+                                   "phases, one copy of the decision device -> host; the host synchronises after every step"},
             "phases": {"draft_us_per_draft_step": draft_us, "draft_us_per_layer": draft_us / wl.d_layers,
                        "draft_kv_gbs": d_gbs, "draft_frac_of_8tbs": d_gbs / 8000.0, "draft_frac_of_measured": d_gbs / peak,
                        "draft_kv_bytes_per_step": draft_bytes_step,
