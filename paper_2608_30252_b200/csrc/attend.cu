@@ -289,6 +289,9 @@ static int draft_attend_impl(masw_mem* mem, int layer, const void* k_raw, const 
   if (n_q * mem->G <= 8) {
     // a slot row whose slot was written by mem_update (not by this launch) reads that entry: never ahead of the wait
     p.early = (mem->kv_clean && !(last_row_is_slot && slot.h_g == nullptr)) ? 1 : 0;
+    // a launch that must wait first may still ask its tiles into L2 early, if they will still be there when it runs
+    const long long kv_bytes = 4LL * entries_upper * c.batch * c.n_kv_heads * c.head_dim;
+    p.guess_hint = (kv_bytes <= (48LL << 20)) ? 1 : 0;
     const int te = (c.head_dim == 64) ? DraftCfg<64>::TE : DraftCfg<128>::TE;   // equals tile_entries(head_dim, 1): same tensor maps
     const int tiles_upper = (entries_upper + te - 1) / te + 4;
     // at most four rows: the instance that packs both bf16 terms of the probabilities into one MMA's columns

@@ -516,8 +516,10 @@ attend_draft_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     // The launch in front may still be writing the counters (a counter update, a rollback) or the arena, so
     // nothing is READ for use ahead of the wait.  But this CTA's tiles can be asked into L2 from a guess: the
     // counters as they stand now (one step old at worst) name almost the same entries, a prefetch returns no
-    // data, and a wrong guess costs nothing but the hint.  The real plan follows behind the wait.
-    if (is_producer) {
+    // data, and a wrong guess costs nothing but the hint.  The real plan follows behind the wait.  (Only where the
+    // launch's KV is small beside L2: at batch 16 the predecessor streams twice the L2's size past the hinted
+    // lines before they are used, and the hint then cost 6 % of the launch.)
+    if (is_producer && p.guess_hint) {
       Segment seg[kMaxSeg];
       int t_g, m_g;
       const int nseg_g = build_segments<true>(p, b, seg, t_g, m_g);

@@ -66,6 +66,8 @@ struct AttendParams {
                            // the launch's immediate predecessor in the stream, so they may be read before the wait
   int deterministic;       // verify (tcgen05 kernel): every tile assigned statically, results repeat bit for bit
   int next_hint;           // verify (tcgen05 kernel): the second pair of tensor maps names the next call's cache (L2 hint)
+  int guess_hint;          // draft (attend_draft_kernel), launch that may not run ahead: ask the tiles into L2 ahead of the
+                           // wait from the counters as they stand (set when the launch's KV is small beside L2)
 #ifdef MASW_TRACE
   long long* trace;        // developer build: per-CTA phase timestamps (null = off)
   int drop_tile;           // developer build: the copy of this CTA-local tile is armed but never issued (-1 = off),

@@ -202,6 +202,16 @@ static MemGeom geom_of(const masw_mem* m) {
   return MemGeom{m->cfg.batch, m->cfg.n_kv_heads, m->cfg.head_dim, m->cfg.sink, m->cfg.max_slots, m->ring_cap, m->n_cap};
 }
 
+// The counter kernels let their successor be set up early only where that pays: the successor's CTAs then sit
+// beside the still running attention launch, and at large batch (a bandwidth- and issue-bound launch of hundreds
+// of MB) that cost 5 % of the launch, while a batch-1 decode step gains a little.  Same size rule as the
+// attention launch's own early L2 hint.
+static int counters_overlap(const masw_mem* m) {
+  const masw_config& c = m->cfg;
+  const long long entries = c.sink + std::min(m->slots_upper + 1, c.max_slots) + c.window;
+  return (4LL * entries * c.batch * c.n_kv_heads * c.head_dim <= (48LL << 20)) ? 1 : 0;
+}
+
 }  // namespace masw
 
 using namespace masw;
@@ -403,7 +413,7 @@ extern "C" int mem_advance(masw_mem* mem, int n_tokens, int add_slot, const uint
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = counters_overlap(mem);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, advance_kernel, mem->d_t, mem->d_slots, mem->d_status, active, B, n_tokens,
@@ -426,7 +436,7 @@ extern "C" int mem_rollback(masw_mem* mem, const int32_t* t_keep, const int32_t*
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = counters_overlap(mem);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, rollback_kernel, mem->d_t, mem->d_slots, t_keep, slots_keep, B));
