@@ -166,6 +166,27 @@ def test_boundary_step_in_one_launch():
     q.check_state()
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_every_instance_of_the_decode_kernel(D):
+    """The decode kernel is compiled per (head_dim, packed probability terms or not, slot materialisation or not).
+    Groups of one, two and four heads with one to three pending tokens put one to eight rows on a KV head, so that
+    every instance runs: rows of different tokens (different visibility bounds) inside the packed instance, the
+    packed instance with the fused slot (group of two: raw row + slot row = four rows), the unpacked ones beside
+    them; ragged batch, sinks, ring wrap, the stored slot read back and attended over by later steps."""
+    seed = 40 + D
+    for Hq, Hkv, n_raw, steps in ((2, 2, 1, 60), (2, 2, 3, 30), (4, 2, 1, 80), (4, 2, 2, 40), (4, 2, 3, 30), (8, 2, 1, 60)):
+        p = Pair(inputs.rng_for(6, 0, seed), L=1, B=2, Hq=Hq, Hkv=Hkv, D=D, S=3, W=20, r=2 * n_raw, max_slots=96, gamma_max=3,
+                 rollback=4, d_model=128)
+        seed += 1
+        p.o.t[1] = n_raw
+        p.o.raw[0][1] = [(np.zeros((Hkv, D)), np.zeros((Hkv, D)))] * n_raw
+        p.g.mem_set_state(t=[0, n_raw], n_slots=[0, 0])
+        for i in range(steps):
+            p.step(n_raw=n_raw, fused=True, fused_slot=(i % 3 != 0))
+        p.check_state()
+        assert p.worst[1] < 1e-4, (Hq, Hkv, n_raw, p.worst)   # both bf16 terms of the probabilities are in the result
+
+
 def test_multi_token_pending_rows_and_slot_row():
     """n_raw > 1 pending tokens per call (causal among themselves) with the slot row riding on the last."""
     p = Pair(inputs.rng_for(6, 0, 2), L=1, B=1, Hq=8, Hkv=2, D=64, S=3, W=10, r=3, max_slots=64, gamma_max=3, rollback=4)
