@@ -182,7 +182,9 @@ class StepRunner:
                                               out=self.d_o2[l], lse=self.d_lse2[l])
                 else:
                     mem.draft_append_attend(l, k[l], v[l], q[l], out=self.d_o1[l], lse=self.d_lse1[l])
-            mem.mem_advance(1, add_slot=fire)
+            # noted on the host only: the launches that follow and the rollback take it as launch parameters, so no
+            # counter kernel sits between draft steps and the next step's first layer may run ahead like the others
+            mem.mem_advance(1, add_slot=fire, deferred=True)
 
     def verify_phase(self):
         wl = self.wl

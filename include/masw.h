@@ -173,6 +173,24 @@ int mem_update(masw_mem* mem, int layer, const void* k_raw, const void* v_raw, i
  * n_slots[b] += 1 for every sequence with active[b] != 0 (active [device] or NULL = all). */
 int mem_advance(masw_mem* mem, int n_tokens, int add_slot, const uint8_t* active, void* stream);
 
+/* The same counter update for all sequences (no `active` mask), noted on the host only: nothing is launched
+ * and nothing on the device changes.  The draft attention calls that follow and mem_rollback take the noted
+ * amounts as launch parameters (t[b] + pending tokens, min(n_slots[b] + pending slots, max_slots) are the
+ * counters in force); every other call that reads or writes the counters (mem_get_state, mem_set_state,
+ * mem_update, mem_load, mem_advance, draft_prefill_attend) first applies them with one launch, as mem_flush
+ * does.  What it buys (Section 4.3: the draft runs L_draft steps back to back): no counter kernel between
+ * draft steps, and the first layer's launch of the next step may run ahead of its predecessor like any other
+ * layer's, because no launch in between writes the counters.  Several deferred updates accumulate.
+ * CUDA graphs: the amounts are baked into the launches that are recorded after this call, so a graph must
+ * contain the whole span from the first deferred update to the call that applies it (mem_rollback,
+ * mem_flush, ...), and the handle must have nothing pending when the recording starts.
+ * Returns MASW_ECAPACITY if the host-side bound on the slot count says the region is full; a slot count that
+ * would exceed max_slots on the device is clamped and reported (MASW_STATUS_SLOT_OVERFLOW) when applied. */
+int mem_advance_deferred(masw_mem* mem, int n_tokens, int add_slot);
+
+/* Applies what mem_advance_deferred noted (one small launch on `stream`; nothing when nothing is pending). */
+int mem_flush(masw_mem* mem, void* stream);
+
 /* Section 4.3, "Rollback": after a rejection drop the speculative raw tokens and the slots created
  * after the last accepted position.  t_keep, slots_keep [device] int32 [batch]: the new counters
  * (t_keep[b] <= t[b], not more than `rollback` + gamma_max tokens back; slots_keep[b] <= n_slots[b]).

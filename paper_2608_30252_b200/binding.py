@@ -22,7 +22,7 @@ KV_STABLE = 2
 
 EXPORTED_SYMBOLS = [
     "masw_sizes", "mem_init", "mem_free", "mem_load", "mem_set_state", "mem_get_state", "mem_update",
-    "mem_advance", "mem_rollback", "draft_attend", "draft_append_attend", "draft_boundary_attend", "draft_prefill_slots",
+    "mem_advance", "mem_advance_deferred", "mem_flush", "mem_rollback", "draft_attend", "draft_append_attend", "draft_boundary_attend", "draft_prefill_slots",
     "draft_prefill_attend", "verify_workspace_bytes", "verify_attend", "verify_paged_workspace_bytes", "verify_attend_paged",
     "verify_fp8_workspace_bytes", "verify_attend_fp8",
     "accept_workspace_bytes", "accept_reject", "accept_reject_static", "masw_last_error", "masw_launch_count", "masw_version",
@@ -75,6 +75,8 @@ def _open(path) -> C.CDLL:
     lib.mem_get_state.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.mem_update.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     lib.mem_advance.argtypes = [vp, i32, i32, vp, vp]
+    lib.mem_advance_deferred.argtypes = [vp, i32, i32]
+    lib.mem_flush.argtypes = [vp, vp]
     lib.mem_rollback.argtypes = [vp, vp, vp, i32, vp]
     lib.draft_attend.argtypes = [vp, i32, vp, i32, i32, vp, vp, vp, vp]
     lib.draft_append_attend.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp]
@@ -92,6 +94,7 @@ def _open(path) -> C.CDLL:
     lib.masw_launch_count.restype = C.c_uint64
     lib.masw_version.restype = C.c_char_p
     for name in ("masw_sizes", "mem_init", "mem_load", "mem_set_state", "mem_get_state", "mem_update", "mem_advance",
+                 "mem_advance_deferred", "mem_flush",
                  "mem_rollback", "draft_attend", "draft_append_attend", "draft_boundary_attend", "verify_attend", "accept_reject"):
         getattr(lib, name).restype = C.c_int
     return lib
@@ -214,8 +217,15 @@ class DraftMemory:
         _check(self.lib.mem_update(self.handle, layer, _ptr(k_raw), _ptr(v_raw), n_raw, _ptr(h_g), _ptr(Wk_g),
                                    _ptr(Wv_g), _ptr(slot_pos), _ptr(active), _stream()))
 
-    def mem_advance(self, n_tokens, add_slot=False, active=None):
-        _check(self.lib.mem_advance(self.handle, n_tokens, 1 if add_slot else 0, _ptr(active), _stream()))
+    def mem_advance(self, n_tokens, add_slot=False, active=None, deferred=False):
+        if deferred:
+            assert active is None, "a deferred counter update applies to all sequences"
+            _check(self.lib.mem_advance_deferred(self.handle, n_tokens, 1 if add_slot else 0))
+        else:
+            _check(self.lib.mem_advance(self.handle, n_tokens, 1 if add_slot else 0, _ptr(active), _stream()))
+
+    def mem_flush(self):
+        _check(self.lib.mem_flush(self.handle, _stream()))
 
     def mem_rollback(self, t_keep, slots_keep, slots_keep_max=-1):
         assert t_keep.dtype == torch.int32 and slots_keep.dtype == torch.int32

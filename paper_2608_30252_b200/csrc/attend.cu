@@ -276,6 +276,7 @@ static int draft_attend_impl(masw_mem* mem, int layer, const void* k_raw, const 
   p.part_o = mem->d_part_o; p.part_ml = mem->d_part_ml;
   p.tickets = mem->d_tickets_attn; p.status = mem->d_status;
   p.t = mem->d_t; p.n_slots = mem->d_slots; p.kv_len = nullptr;
+  p.dt = mem->pend_t; p.dm = mem->pend_m;   // a deferred counter update travels as launch parameters
   p.n_q = n_q; p.last_row_is_slot = last_row_is_slot;
   p.G = mem->G; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads;
   p.S = c.sink; p.W = c.window; p.ring_cap = mem->ring_cap; p.max_slots = c.max_slots;

@@ -206,7 +206,7 @@ __device__ __forceinline__ void draft_reduce_and_store(const AttendParams& p, in
       if (lane == 0) sg[warp] = dot * p.scale_log2e;
     }
     if (split == 0) {
-      const int m_slot = p.n_slots[b];
+      const int m_slot = p.n_slots[b] + p.dm;
       if (m_slot < p.max_slots) {
         for (int c = tid; c < 2 * D; c += NT) {
           __nv_bfloat16* dst = (c < D ? p.k_base : p.v_base) + b * p.stride_b + kvh * p.stride_h +

@@ -66,6 +66,8 @@ struct AttendParams {
                            // the launch's immediate predecessor in the stream, so they may be read before the wait
   int deterministic;       // verify (tcgen05 kernel): every tile assigned statically, results repeat bit for bit
   int next_hint;           // verify (tcgen05 kernel): the second pair of tensor maps names the next call's cache (L2 hint)
+  int dt, dm;              // draft: a counter update that was only noted on the host (mem_advance_deferred): the counters in
+                           // force are t[b] + dt and min(n_slots[b] + dm, max_slots)
   int guess_hint;          // draft (attend_draft_kernel), launch that may not run ahead: ask the tiles into L2 ahead of the
                            // wait from the counters as they stand (set when the launch's KV is small beside L2)
 #ifdef MASW_TRACE
@@ -107,8 +109,8 @@ __device__ __forceinline__ int build_segments(const AttendParams& p, int b, Segm
     if (len > 0) seg[n++] = Segment{0, len, 0, 2};
     return n;
   }
-  const int t = max(ld_counter(p.t + b, HINT), 0);
-  const int M = min(max(ld_counter(p.n_slots + b, HINT), 0), p.max_slots);
+  const int t = max(ld_counter(p.t + b, HINT), 0) + p.dt;
+  const int M = min(max(ld_counter(p.n_slots + b, HINT), 0) + p.dm, p.max_slots);
   t_out = t;
   m_out = M;
   const int n_raw = p.n_q - p.last_row_is_slot;
@@ -305,7 +307,7 @@ __device__ __forceinline__ void split_reduce_and_store(const AttendParams& p, in
         if (lane == 0) sg[g] = dot * p.scale_log2e;
       }
       if (split == 0) {
-        const int m_slot = p.n_slots[b];
+        const int m_slot = p.n_slots[b] + p.dm;
         if (m_slot < p.max_slots) {
           for (int c = tid; c < 2 * D; c += NTHREADS) {
             __nv_bfloat16* dst = (c < D ? p.k_base : p.v_base) + b * p.stride_b + kvh * p.stride_h +

@@ -167,19 +167,22 @@ __global__ void advance_kernel(int* t, int* n_slots, int* status, const uint8_t*
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   t[b] += n_tokens;
-  if (add_slot && (active == nullptr || active[b] != 0)) {
-    if (n_slots[b] < max_slots) n_slots[b] += 1;
-    else if (status) atomicOr(status, MASW_STATUS_SLOT_OVERFLOW);
+  if (add_slot && (active == nullptr || active[b] != 0)) {   // add_slot: how many slots were committed (one, or several deferred)
+    const int m = n_slots[b] + add_slot;
+    n_slots[b] = min(m, max_slots);
+    if (m > max_slots && status) atomicOr(status, MASW_STATUS_SLOT_OVERFLOW);
   }
 }
 
-__global__ void rollback_kernel(int* t, int* n_slots, const int* t_keep, const int* slots_keep, int B) {
+__global__ void rollback_kernel(int* t, int* n_slots, const int* t_keep, const int* slots_keep, int B, int pend_t, int pend_m,
+                                int max_slots) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // as in advance_kernel
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
-  t[b] = max(0, min(t[b], t_keep[b]));
-  n_slots[b] = max(0, min(n_slots[b], slots_keep[b]));
+  // (pend_t, pend_m): a deferred counter update that this launch applies on the way
+  t[b] = max(0, min(t[b] + pend_t, t_keep[b]));
+  n_slots[b] = max(0, min(min(n_slots[b] + pend_m, max_slots), slots_keep[b]));
 }
 
 static int validate_config(const masw_config* c) {
@@ -210,6 +213,32 @@ static int counters_overlap(const masw_mem* m) {
   const masw_config& c = m->cfg;
   const long long entries = c.sink + std::min(m->slots_upper + 1, c.max_slots) + c.window;
   return (4LL * entries * c.batch * c.n_kv_heads * c.head_dim <= (48LL << 20)) ? 1 : 0;
+}
+
+static int launch_advance(masw_mem* mem, int n_tokens, int add_slots, const uint8_t* active, cudaStream_t st) {
+  const int B = mem->cfg.batch;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((B + 127) / 128, 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = counters_overlap(mem);
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, advance_kernel, mem->d_t, mem->d_slots, mem->d_status, active, B, n_tokens, add_slots,
+                                   mem->cfg.max_slots));
+  count_launch();
+  return MASW_OK;
+}
+
+int flush_counters(masw_mem* mem, cudaStream_t st) {
+  if (mem->pend_t == 0 && mem->pend_m == 0) return MASW_OK;
+  const int dt = mem->pend_t, dm = mem->pend_m;
+  mem->pend_t = 0;
+  mem->pend_m = 0;
+  mem->kv_clean = false;   // the counters are written: the next attention launch reads them behind its wait
+  return launch_advance(mem, dt, dm, nullptr, st);
 }
 
 }  // namespace masw
@@ -285,6 +314,7 @@ extern "C" void mem_free(masw_mem* mem) { delete mem; }
 extern "C" int mem_load(masw_mem* mem, int layer, int region, const void* k, const void* v, int first, int n,
                         const int64_t strides[3], void* stream) {
   MASW_REQUIRE(mem != nullptr && k != nullptr && v != nullptr && strides != nullptr, MASW_EINVAL, "mem_load: null argument");
+  { const int rc = flush_counters(mem, static_cast<cudaStream_t>(stream)); if (rc != MASW_OK) return rc; }
   mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   MASW_REQUIRE(layer >= 0 && layer < mem->cfg.n_layers, MASW_EINVAL, "mem_load: layer %d out of range", layer);
   MASW_REQUIRE(n >= 0 && first >= 0, MASW_EINVAL, "mem_load: negative count or index");
@@ -314,6 +344,7 @@ extern "C" int mem_load(masw_mem* mem, int layer, int region, const void* k, con
 
 extern "C" int mem_set_state(masw_mem* mem, const int32_t* t, const int32_t* n_slots, void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_set_state: null handle");
+  { const int rc = flush_counters(mem, static_cast<cudaStream_t>(stream)); if (rc != MASW_OK) return rc; }
   mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   const int B = mem->cfg.batch;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -336,6 +367,7 @@ extern "C" int mem_set_state(masw_mem* mem, const int32_t* t, const int32_t* n_s
 
 extern "C" int mem_get_state(masw_mem* mem, int32_t* t, int32_t* n_slots, int32_t* status, void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_get_state: null handle");
+  { const int rc = flush_counters(mem, static_cast<cudaStream_t>(stream)); if (rc != MASW_OK) return rc; }
   const int B = mem->cfg.batch;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (t) MASW_CUDA_TRY(cudaMemcpyAsync(t, mem->d_t, sizeof(int) * B, cudaMemcpyDeviceToHost, st));
@@ -352,6 +384,7 @@ extern "C" int mem_update(masw_mem* mem, int layer, const void* k_raw, const voi
                           const void* Wk_g, const void* Wv_g, const int32_t* slot_pos, const uint8_t* active,
                           void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_update: null handle");
+  { const int rc = flush_counters(mem, static_cast<cudaStream_t>(stream)); if (rc != MASW_OK) return rc; }
   mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   MASW_REQUIRE(layer >= 0 && layer < mem->cfg.n_layers, MASW_EINVAL, "mem_update: layer %d out of range", layer);
   const masw_config& c = mem->cfg;
@@ -399,28 +432,32 @@ extern "C" int mem_update(masw_mem* mem, int layer, const void* k_raw, const voi
 
 extern "C" int mem_advance(masw_mem* mem, int n_tokens, int add_slot, const uint8_t* active, void* stream) {
   MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_advance: null handle");
-  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   MASW_REQUIRE(n_tokens >= 0 && n_tokens <= mem->cfg.gamma_max, MASW_EINVAL, "mem_advance: n_tokens %d outside [0, gamma_max]", n_tokens);
+  { const int rc = flush_counters(mem, static_cast<cudaStream_t>(stream)); if (rc != MASW_OK) return rc; }
+  mem->kv_clean = false;   // this call writes the counters or the arena: the next attention launch reads them behind its wait
   if (add_slot) {
     MASW_REQUIRE(mem->slots_upper < mem->cfg.max_slots, MASW_ECAPACITY, "mem_advance: slot region full");
     mem->slots_upper += 1;
   }
-  const int B = mem->cfg.batch;
-  {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((B + 127) / 128, 1, 1);
-    cfg.blockDim = dim3(128, 1, 1);
-    cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = counters_overlap(mem);
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, advance_kernel, mem->d_t, mem->d_slots, mem->d_status, active, B, n_tokens,
-                                     add_slot ? 1 : 0, mem->cfg.max_slots));
+  return launch_advance(mem, n_tokens, add_slot ? 1 : 0, active, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int mem_advance_deferred(masw_mem* mem, int n_tokens, int add_slot) {
+  MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_advance_deferred: null handle");
+  MASW_REQUIRE(n_tokens >= 0 && n_tokens <= mem->cfg.gamma_max, MASW_EINVAL, "mem_advance_deferred: n_tokens %d outside [0, gamma_max]",
+               n_tokens);
+  if (add_slot) {
+    MASW_REQUIRE(mem->slots_upper < mem->cfg.max_slots, MASW_ECAPACITY, "mem_advance_deferred: slot region full");
+    mem->slots_upper += 1;
+    mem->pend_m += 1;
   }
-  count_launch();
+  mem->pend_t += n_tokens;   // nothing is launched and nothing on the device changes: kv_clean stays as it is
   return MASW_OK;
+}
+
+extern "C" int mem_flush(masw_mem* mem, void* stream) {
+  MASW_REQUIRE(mem != nullptr, MASW_EINVAL, "mem_flush: null handle");
+  return flush_counters(mem, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int mem_rollback(masw_mem* mem, const int32_t* t_keep, const int32_t* slots_keep, int slots_keep_max,
@@ -439,8 +476,11 @@ extern "C" int mem_rollback(masw_mem* mem, const int32_t* t_keep, const int32_t*
     attr[0].val.programmaticStreamSerializationAllowed = counters_overlap(mem);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, rollback_kernel, mem->d_t, mem->d_slots, t_keep, slots_keep, B));
+    MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, rollback_kernel, mem->d_t, mem->d_slots, t_keep, slots_keep, B, mem->pend_t, mem->pend_m,
+                                     mem->cfg.max_slots));
   }
+  mem->pend_t = 0;   // a deferred counter update was applied by this launch
+  mem->pend_m = 0;
   count_launch();
   return MASW_OK;
 }

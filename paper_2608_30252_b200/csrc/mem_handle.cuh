@@ -83,9 +83,18 @@ struct masw_mem {
   // or the arena through another path (mem_update, mem_load, mem_advance, mem_rollback, mem_set_state, the
   // prefill import) clears it.
   bool kv_clean = false;
+  // A counter update that was only noted (mem_advance_deferred): t[b] + pend_t and min(n_slots[b] + pend_m,
+  // max_slots) are the counters in force.  Draft attention launches and mem_rollback take the two numbers as
+  // launch parameters; every other call that reads or writes the counters applies them first (flush_counters).
+  int pend_t = 0, pend_m = 0;
 
   __nv_bfloat16* k_layer(int layer) const {
     return reinterpret_cast<__nv_bfloat16*>(arena) + static_cast<size_t>(layer) * 2 * tensor_elems;
   }
   __nv_bfloat16* v_layer(int layer) const { return k_layer(layer) + tensor_elems; }
 };
+
+namespace masw {
+// Applies a deferred counter update with one launch of the advance kernel (no-op when nothing is pending).
+int flush_counters(masw_mem* mem, cudaStream_t st);
+}  // namespace masw

@@ -45,6 +45,7 @@ extern "C" int draft_prefill_slots(const masw_config* cfg, int P) {
 extern "C" int draft_prefill_attend(masw_mem* mem, int layer, const masw_kv_desc* kv, const void* q, int P, float* o,
                                     float* lse, void* o_bf16, int import_memory, void* stream) {
   MASW_REQUIRE(mem != nullptr && kv != nullptr && q != nullptr, MASW_EINVAL, "draft_prefill_attend: null argument");
+  { const int rc = flush_counters(mem, static_cast<cudaStream_t>(stream)); if (rc != MASW_OK) return rc; }
   mem->kv_clean = false;   // the import writes the arena
   MASW_REQUIRE(o != nullptr || o_bf16 != nullptr, MASW_EINVAL, "draft_prefill_attend: one of o, o_bf16 must be given");
   MASW_REQUIRE(kv->k != nullptr && kv->v != nullptr, MASW_EINVAL, "draft_prefill_attend: null K/V pointer");

@@ -111,7 +111,7 @@ class ToyDraft:
         else:
             q = (x @ self.Wq).view(1, -1, self.Hq, self.D).to(torch.bfloat16).contiguous()
             o, _ = self.mem.draft_append_attend(0, k, v, q)
-        self.mem.mem_advance(n, add_slot=boundary)
+        self.mem.mem_advance(n, add_slot=boundary, deferred=True)   # applied by the next rollback (or state read)
         self.t = t_after
         self.slots += int(boundary)
         logits = o[0, n - 1].reshape(-1) @ self.Wu

@@ -28,6 +28,7 @@ class Pair:
         self.dWv = [dev_bf16(w) for w in self.Wv]
         self.worst = (0.0, 0.0)
         self.slot_ulps = 0
+        self.deferred = False   # counter updates noted on the host only (mem_advance_deferred)
 
     def step(self, n_raw=1, check=True, q_scale=1.0, fused=False, fused_slot=False):
         o, rng = self.o, self.rng
@@ -85,7 +86,11 @@ class Pair:
                 mx, rel = assert_attention_close(og.cpu().numpy(), oref, lg.cpu().numpy(), lref, tag=f"t={o.t} l={l}")
                 self.worst = (max(self.worst[0], mx), max(self.worst[1], rel))
         o.advance(n_raw, slot_added=boundary)
-        self.g.mem_advance(n_raw, add_slot=fire, active=act)
+        if self.deferred:
+            assert all(boundary) == any(boundary)   # a deferred update has no per-sequence mask
+            self.g.mem_advance(n_raw, add_slot=fire, deferred=True)
+        else:
+            self.g.mem_advance(n_raw, add_slot=fire, active=act)
 
     def check_state(self):
         t, m, status = self.g.mem_get_state()
@@ -349,6 +354,34 @@ def test_rollback_reexposes_window_and_drops_slots():
     for _ in range(10):                     # decoding continues from the restored state
         p.step()
     p.check_state()
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_deferred_counter_updates(D):
+    """mem_advance_deferred notes the counter update on the host; the attention launches that follow and the
+    rollback take it as launch parameters, every other call applies it first.  Speculative blocks of four draft
+    steps (fused append, fused slot materialisation in the block) with nothing but attention launches between
+    them, then a rollback that keeps 0..4 of the tokens (Section 4.3, "Rollback"); the counters are read back
+    every other block (which applies what is pending), an unfused mem_update joins in now and then, and every
+    attention output is checked against the oracle."""
+    p = Pair(inputs.rng_for(6, 0, 70 + D), L=2, B=2, Hq=8, Hkv=2, D=D, S=3, W=24, r=4, max_slots=96, rollback=8, d_model=128)
+    p.deferred = True
+    for block in range(24):
+        t_keep, m_keep = list(p.o.t), list(p.o.M)
+        for j in range(4):
+            p.step(fused=(block % 5 != 4), fused_slot=True)
+        keep = block % 5
+        if keep < 4:
+            t_new = [t + keep for t in t_keep]
+            m_new = [max(0, t - 3) // 4 for t in t_new]
+            p.o.rollback(t_new, m_new)
+            p.g.mem_rollback(torch.tensor(t_new, dtype=torch.int32, device="cuda"),
+                             torch.tensor(m_new, dtype=torch.int32, device="cuda"), slots_keep_max=max(m_new))
+        if block % 2 == 0:
+            p.check_state()
+    p.g.mem_flush()
+    p.check_state()
+    assert p.worst[1] < 2e-3
 
 
 def test_slot_region_overflow_is_reported_not_written():
