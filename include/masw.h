@@ -110,10 +110,11 @@ enum {
    * because every split waits for the slowest SM. */
   MASW_KV_DETERMINISTIC = 1,
   /* verify_attend, head_dim 128, contiguous cache: the caller vouches that the kernel which precedes this call
-   * in the stream writes nothing of the K and V arrays (the T new rows were appended by an earlier kernel, or
-   * the cache is static as in a benchmark).  The launch may then request its first K/V tiles before it waits
-   * for that kernel; q, kv_len and the scratch are still read behind the wait.  Without the flag everything is
-   * read behind the wait. */
+   * in the stream writes nothing of the K and V arrays nor of kv_len (the T new rows were appended and the
+   * lengths set by an earlier kernel, as they are for every layer but the first of a verification pass, or the
+   * cache is static as in a benchmark).  The launch may then read kv_len and request its first K/V tiles (a
+   * whole ring of them) before it waits for that kernel; q and the scratch are still read behind the wait.
+   * Without the flag everything is read behind the wait. */
   MASW_KV_STABLE = 2
 };
 

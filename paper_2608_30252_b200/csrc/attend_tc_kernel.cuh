@@ -309,7 +309,28 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     n_early = 1;
     first_requested = true;
   };
-  if (tid == 0 && p.early && p.page_table == nullptr) request_first_tile();
+  // The tile schedule behind the first tile depends on the cache length alone (see the plan below).
+  auto plan_schedule = [&](int len) {
+    const int nt = (len + C::kTile - 1) / C::kTile;
+    const int rest = max(0, nt - p.splits);
+    if (p.deterministic) {
+      const int base = rest / p.splits, rem = rest % p.splits;
+      n_static = base + (split < rem ? 1 : 0);
+      n_pool = 0;
+      static_first = p.splits + split * base + min(split, rem);
+    } else {
+      n_static = (rest * kStaticNum / kStaticDen) / p.splits;
+      n_pool = rest - n_static * p.splits;
+      static_first = p.splits + n_pool + split * n_static;
+    }
+  };
+  int len_early = -1;   // a stable cache includes its length: read ahead of the wait
+  if (tid == 0 && p.early && p.page_table == nullptr) {
+    request_first_tile();
+    if (!FP8 && NQ == 32) {   // (the 64-row instance is bound by its softmax loop: there the early requests gained nothing)
+      len_early = min(max(__ldg(p.kv_len + b), 0), p.capacity);
+    }
+  }
   // nothing else above touched global memory: a launch that was allowed to start early waits here for its
   // predecessor, and lets its own successor be set up
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -334,9 +355,29 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   }
   const int len_raw = (tid < NQ) ? __ldg(p.kv_len + b) : 0;
   const int epoch_raw = (tid == 0) ? __ldcg(p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1)) : 0;
+  if (tid == 0 && len_early >= 0) {
+    // The rest of the K and V rings (this CTA's first static tiles) is requested now, behind the Q loads in the
+    // queues but without waiting for them: the prologue's own loads take about 2 us behind the launch's burst of
+    // first tiles, and HBM has little else to do meanwhile.
+    plan_schedule(len_early);
+    const uint64_t policy = l2_policy_evict_first();
+    const int n_pre = min((NK < NV ? NK : NV) - 1, n_static);
+    for (int i = 1; i <= n_pre; ++i) {
+      const int row0 = (static_first + i - 1) * C::kTile;
+      uint8_t* kdst = k_ring + i * C::kTileBytes;
+      uint8_t* vdst = v_ring + i * C::kTileBytes;
+      mbar_arrive_expect_tx(&ctl->k_full[i], C::kTileBytes);
+      tma_load_4d(kdst, &tmK, &ctl->k_full[i], 0, row0, kvh, b, policy);
+      tma_load_4d(kdst + C::kSubBytes, &tmK, &ctl->k_full[i], 64, row0, kvh, b, policy);
+      mbar_arrive_expect_tx(&ctl->v_full[i], C::kTileBytes);
+      tma_load_4d(vdst, &tmV, &ctl->v_full[i], 0, row0, kvh, b, policy);
+      tma_load_4d(vdst + C::kSubBytes, &tmV, &ctl->v_full[i], 64, row0, kvh, b, policy);
+      ctl->tile_id[i] = static_first + i - 1;
+    }
+    n_early = 1 + n_pre;
+  }
   if (tid == 0) {
     const int len = min(max(len_raw, 0), p.capacity);
-    const int nt = (len + C::kTile - 1) / C::kTile;
     // Tile schedule of the tiles behind the first `splits` ones.  A quarter of them is assigned statically
     // (n_static consecutive tiles per split, at the end of the cache, so that the ragged and masked last tile
     // is never the last one a CTA meets); the others form a pool from which the splits of this (sequence,
@@ -346,17 +387,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // In the deterministic mode there is no pool: every tile is assigned statically (the remainder goes to the
     // first splits), so each split meets the same tiles in the same order in every launch and the result
     // repeats bit for bit, at the price of waiting for the slowest SM.
-    const int rest = max(0, nt - p.splits);
-    if (p.deterministic) {
-      const int base = rest / p.splits, rem = rest % p.splits;
-      n_static = base + (split < rem ? 1 : 0);
-      n_pool = 0;
-      static_first = p.splits + split * base + min(split, rem);
-    } else {
-      n_static = (rest * kStaticNum / kStaticDen) / p.splits;
-      n_pool = rest - n_static * p.splits;
-      static_first = p.splits + n_pool + split * n_static;
-    }
+    plan_schedule(len);
     const int epoch = epoch_raw;
     pool_ctr = p.tickets + (b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + (epoch & 1);
     pending = (n_pool > 0) ? atomicAdd(pool_ctr, 1) : 0x7fffffff;   // used only after the static tiles
