@@ -282,7 +282,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   // request goes out before the wait: a CTA that starts while the predecessor's last CTAs are still draining
   // then has its first tile on the way when the wait ends.
   bool first_requested = false;
-  auto request_first_tile = [&]() {
+  auto request_first_tile = [&](bool with_v = true) {
     const uint64_t policy = l2_policy_evict_first();
     // contiguous cache: tile t of sequence b starts at entry 128 t; paged cache: it is page page_table[b][t]
     // of the pool (the map's outermost coordinate), entries 0..127 of that page
@@ -301,9 +301,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       mbar_arrive_expect_tx(&ctl->k_full[0], C::kTileBytes);
       tma_load_4d(k_ring, &tmK, &ctl->k_full[0], 0, row0, kvh, outer, policy);
       tma_load_4d(k_ring + C::kSubBytes, &tmK, &ctl->k_full[0], 64, row0, kvh, outer, policy);
-      mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
-      tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, row0, kvh, outer, policy);
-      tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, row0, kvh, outer, policy);
+      if (with_v) {
+        mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
+        tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, row0, kvh, outer, policy);
+        tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, row0, kvh, outer, policy);
+      }
     }
     ctl->tile_id[0] = split;
     n_early = 1;
@@ -326,10 +328,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   };
   int len_early = -1;   // a stable cache includes its length: read ahead of the wait
   if (tid == 0 && p.early && p.page_table == nullptr) {
-    request_first_tile();
-    if (!FP8 && NQ == 32) {   // (the 64-row instance is bound by its softmax loop: there the early requests gained nothing)
-      len_early = min(max(__ldg(p.kv_len + b), 0), p.capacity);
-    }
+    constexpr bool kRingEarly = !FP8 && NQ == 32;   // (the 64-row instance is bound by its softmax loop: there the early requests gained nothing)
+    request_first_tile(!kRingEarly);   // ring early: only K goes out here, the first V tile follows the Q loads (it is needed a tile later)
+    if (kRingEarly) len_early = min(max(__ldg(p.kv_len + b), 0), p.capacity);
   }
   // nothing else above touched global memory: a launch that was allowed to start early waits here for its
   // predecessor, and lets its own successor be set up
@@ -361,6 +362,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // first tiles, and HBM has little else to do meanwhile.
     plan_schedule(len_early);
     const uint64_t policy = l2_policy_evict_first();
+    mbar_arrive_expect_tx(&ctl->v_full[0], C::kTileBytes);
+    tma_load_4d(v_ring, &tmV, &ctl->v_full[0], 0, split * C::kTile, kvh, b, policy);
+    tma_load_4d(v_ring + C::kSubBytes, &tmV, &ctl->v_full[0], 64, split * C::kTile, kvh, b, policy);
     const int n_pre = min((NK < NV ? NK : NV) - 1, n_static);
     for (int i = 1; i <= n_pre; ++i) {
       const int row0 = (static_first + i - 1) * C::kTile;
