@@ -141,6 +141,10 @@ accept_reject_kernel(const unsigned short* tl, const unsigned short* dl, const i
   __shared__ int sh_int;
   __shared__ int sh_last;
 
+  // launched with programmatic stream serialisation (accept_reject): the blocks may be set up while the kernel in
+  // front still runs; nothing is read before it has completed, and the successor may be set up at once
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int i = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x;
   const bool sampling = temperature > 0.f;
@@ -314,13 +318,22 @@ extern "C" int accept_reject(const void* target_logits, const void* draft_logits
   const AcceptWs w = accept_ws(batch, gamma);
   MASW_REQUIRE(workspace_bytes >= w.total, MASW_ECAPACITY, "accept_reject: workspace %zu < %zu bytes", workspace_bytes, w.total);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  dim3 grid(gamma + 1, batch);
-  accept_reject_kernel<<<grid, kAcceptThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const unsigned short*>(target_logits), static_cast<const unsigned short*>(draft_logits), draft_tokens,
-      uniforms, gamma, vocab, temperature, n_accepted, out_tokens, status, reinterpret_cast<int*>(ws + w.off_tickets),
-      reinterpret_cast<RowInfo*>(ws + w.off_rows));
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(gamma + 1, batch, 1);
+    cfg.blockDim = dim3(kAcceptThreads, 1, 1);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MASW_CUDA_TRY(cudaLaunchKernelEx(&cfg, accept_reject_kernel, static_cast<const unsigned short*>(target_logits),
+                                     static_cast<const unsigned short*>(draft_logits), draft_tokens, uniforms, gamma, vocab,
+                                     temperature, n_accepted, out_tokens, status, reinterpret_cast<int*>(ws + w.off_tickets),
+                                     reinterpret_cast<RowInfo*>(ws + w.off_rows)));
+  }
   count_launch();
-  MASW_CUDA_TRY(cudaGetLastError());
   return MASW_OK;
 }
 
