@@ -898,8 +898,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   MASW_STAMP(tr, 3);
   // six thread groups per item with three splits' records in flight each: 18 splits in one round trip, and few
   // enough registers that nothing spills
-  static_assert(C::kThreads % (FP8 ? 8 : 6) == 0, "the fetch groups must divide the thread count");
-  split_reduce_and_store<D, NQ, C::kThreads, FP8 ? 8 : 6, 3>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
+  // (the 64-row instance has up to 114 items per CTA: three groups x six records take them in one batch, and its
+  // 168-register cap has room for the eighteen records in flight)
+  constexpr int kRG = FP8 ? 8 : (NQ == 64 ? 3 : 6), kRF = (!FP8 && NQ == 64) ? 6 : 3;
+  static_assert(C::kThreads % kRG == 0, "the fetch groups must divide the thread count");
+  split_reduce_and_store<D, NQ, C::kThreads, kRG, kRF>(p, b, kvh, split, n_rows, ctl->plan[6], reinterpret_cast<float*>(pipe), tid);
   // the pool counter of the next launch (the other parity) is idle now: clear it
   if (split == 0 && tid == 0) p.tickets[(b * p.Hkv + kvh) * (kMaxSplitsDev + 1) + 1 + ((ctl->plan[6] + 1) & 1)] = 0;
   MASW_STAMP(tr, 4);
